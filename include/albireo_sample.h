@@ -1,0 +1,188 @@
+/*
+ * albireo_sample.h -- C ABI of the B200 (sm_100a) batched token sampler.
+ *
+ * The library implements the sampling task T4 of "Albireo" (arxiv 2606.01927, section
+ * 2.1): after every decode step, for each row of the (s x v) logits matrix, choose the
+ * next token.  The paper keeps "the core sampling computation" unchanged (section 6.1,
+ * step 3) and enables every feature in its evaluation (section 8.1, Workload): top-p,
+ * top-k, min-p, temperature, and repetition / presence / frequency penalties driven by
+ * per-sequence metadata (section 3.1, Optimization 3).  Rows are independent (section
+ * 6.1), the result per row is one token id plus its probability (section 6.2, result
+ * gather; Appendix A, "update sequence"), and the draw must not depend on how rows are
+ * partitioned over workers (section 6.2, deterministic random number generation).
+ *
+ * Per row b (global row id R = row_base + b) the library computes, in this order:
+ *   x      = logits widened to fp32
+ *   c_t    = occurrences of token t in the row's history (ids outside [0,V) ignored)
+ *   a_t    = x_t                              if c_t == 0
+ *          = ((x_t > 0 ? x_t / r : x_t * r) - f * c_t) - p   otherwise (fp32, one rounding per op)
+ *   z_t    = a_t * (1 / T)   (fp32; T <= 0 means greedy: top_k = 1 on a_t, other cuts ignored)
+ *   order  = ids sorted by (z descending, id ascending); -0.0 sorts below +0.0
+ *   top-k  : keep the first min(k, #finite z)          (k <= 0 or k >= V: off)
+ *   min-p  : keep z - z_max >= ln(min_p), at least one (min_p <= 0: off)
+ *   top-p  : smallest prefix whose mass reaches top_p * (mass of the survivors) (top_p >= 1: off)
+ *   logprob: log of the softmax over the final kept set
+ *   draw   : w_t = word (t & 3) of Philox4x32-10(counter = (t >> 2, R, step lo, step hi),
+ *            key = (seed lo, seed hi)); v = (w + 1/2) / 2^32; E = -log1p(-v);
+ *            token = argmax_t (z_t - z_max) - ln E_t   (ties: lowest id)
+ *
+ * All data pointers are DEVICE pointers unless a parameter says "host".  The caller
+ * owns every buffer, including the workspace; the library owns only the opaque handle
+ * (host memory) and never allocates or frees device memory.
+ */
+#ifndef ALBIREO_SAMPLE_H
+#define ALBIREO_SAMPLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct albireo_sampler albireo_sampler_t; /* opaque; created by init, freed by destroy */
+
+enum { ALBIREO_F32 = 0, ALBIREO_BF16 = 1 };
+
+enum {
+    ALBIREO_OK = 0,
+    ALBIREO_EINVAL = -1,       /* bad argument; nothing was launched                     */
+    ALBIREO_ENOMEM = -2,       /* host allocation of the handle failed                   */
+    ALBIREO_ECUDA = -3,        /* a CUDA runtime call failed; see albireo_last_error     */
+    ALBIREO_EUNSUPPORTED = -4  /* shape outside what the kernels support (see limits)    */
+};
+
+/* limits */
+#define ALBIREO_MAX_VOCAB 524288   /* V above this is rejected                            */
+#define ALBIREO_MAX_NUM_TOP 128    /* largest num_top (top-N logprob list)                */
+
+/* bits of out_row_status[b] */
+#define ALBIREO_ROW_GENERAL_PATH 1u  /* informational: row took the multi-pass general path */
+#define ALBIREO_ROW_BAD_PARAM 2u     /* T < 0 or NaN, r <= 0, ...: row treated per the clamps */
+#define ALBIREO_ROW_HISTORY_OVERFLOW 4u /* history did not fit the workspace: penalties skipped */
+
+/* flags of albireo_sample_ext_t.flags */
+#define ALBIREO_FLAG_FORCE_GENERAL 1u /* testing: send every row down the general path     */
+
+/*
+ * Optional arguments of albireo_sample (pass NULL for all defaults).  Zero-initialise,
+ * set struct_size = sizeof(albireo_sample_ext_t), then fill what is needed.
+ */
+typedef struct albireo_sample_ext {
+    uint32_t struct_size;
+    uint32_t flags;
+    int64_t row_stride_elems;  /* elements between rows of logits; 0 means V               */
+    uint32_t row_base;         /* global id of row 0 (keeps draws invariant under row
+                                  sharding, section 6.2)                                   */
+    int32_t num_top;           /* > 0: also return the first min(num_top, kept) entries of
+                                  the kept set in order                                     */
+    int32_t *out_top_ids;      /* [B, num_top] device, padded with -1                       */
+    float *out_top_logprobs;   /* [B, num_top] device, padded with -inf                     */
+    int32_t *out_num_kept;     /* [B] device: size of the final kept set (diagnostic)       */
+    int32_t *out_num_topk;     /* [B] device: size of the set kept by the top-k stage       */
+    int32_t dbg_cap;           /* capacity per row of dbg_topk_ids                          */
+    int32_t *dbg_topk_ids;     /* [B, dbg_cap] device: ids kept by the top-k stage, in no
+                                  particular order, -1 padded; written only for rows whose
+                                  top-k stage keeps <= dbg_cap ids                          */
+    uint32_t *out_row_status;  /* [B] device: ALBIREO_ROW_* bits                            */
+} albireo_sample_ext_t;
+
+/*
+ * Device bytes the caller must provide as `workspace` to albireo_sample_init.
+ * The workspace holds per-row history occurrence counts for rows whose history has more
+ * distinct ids than fit on chip (sized by max_history_total, the largest
+ * history_offsets[B] of any call).  Pure function of its arguments; returns 0 on
+ * nonsensical input (negative sizes).
+ */
+size_t albireo_sample_workspace_bytes(int32_t max_rows, int32_t max_vocab, int64_t max_history_total);
+
+/*
+ * Extra device bytes albireo_sample_host needs after the first
+ * albireo_sample_workspace_bytes(...) bytes of the same workspace (staging copies of
+ * every input and output; logits staged at 4 bytes per element).
+ */
+size_t albireo_sample_host_staging_bytes(int32_t max_rows, int32_t max_vocab, int64_t max_history_total);
+
+/*
+ * Creates a sampler bound to CUDA device `device`.
+ *   workspace / workspace_bytes: caller-owned device memory on that device, 256-byte
+ *     aligned, at least albireo_sample_workspace_bytes(...) long (plus the staging
+ *     bytes if albireo_sample_host will be used); must outlive the handle.
+ * Does not allocate device memory and does not synchronise.  Sets per-device kernel
+ * attributes, so call it before capturing a stream that will use the handle.
+ * Returns ALBIREO_OK and stores the handle in *out, or an error code (then *out = NULL).
+ */
+int albireo_sample_init(albireo_sampler_t **out, int32_t device,
+                        int32_t max_rows, int32_t max_vocab, int64_t max_history_total,
+                        void *workspace, size_t workspace_bytes);
+
+/*
+ * Samples one token per row (section 6.1 step 3: Y = Sample(Pr)).  Enqueues work on
+ * `stream` and returns without synchronising; outputs are valid once the stream
+ * reaches that point.  `device` of the handle must be current.
+ *
+ *   logits        [B, V] row-major (row stride = ext->row_stride_elems or V), dtype
+ *                 ALBIREO_F32 (float) or ALBIREO_BF16 (bfloat16).  Each value finite or
+ *                 -inf, at least one finite per row (NaN / +inf: result unspecified but
+ *                 in range).  Never written.  16-byte aligned rows take the vector path;
+ *                 any element-aligned pointer/stride is accepted.
+ *   temperature, top_p, min_p, repetition_penalty, presence_penalty, frequency_penalty
+ *                 float[B], top_k int32[B]; a NULL array switches the feature off for
+ *                 every row (T = 1, k = 0, top_p = 1, min_p = 0, r = 1, p = 0, f = 0).
+ *   history_ids   int32[history_offsets[B]], history_offsets int32[B + 1] (CSR, first
+ *                 entry 0); both NULL for "no history".  One history drives all three
+ *                 penalties.
+ *   seeds         uint64[B] (NULL: all 0); `step` is the decode iteration.
+ *   out_tokens    int32[B]; out_logprobs float[B] (log-probability of the token under the
+ *                 final kept-set distribution).
+ *   stream        a cudaStream_t passed as void* (NULL: the legacy default stream).
+ *
+ * B = 0 returns ALBIREO_OK without launching.  Errors detectable on the host (NULL
+ * required pointer, B < 0 or > max_rows, V < 1 or > max_vocab, unknown dtype, wrong
+ * current device, bad ext) return ALBIREO_EINVAL / ALBIREO_EUNSUPPORTED with nothing
+ * launched; per-row parameter values live on the device and are clamped as stated above.
+ * One call at a time per handle (the workspace is shared by the rows of one call).
+ */
+int albireo_sample(albireo_sampler_t *h,
+                   const void *logits, int32_t B, int32_t V, int32_t dtype,
+                   const float *temperature, const int32_t *top_k,
+                   const float *top_p, const float *min_p,
+                   const float *repetition_penalty, const float *presence_penalty,
+                   const float *frequency_penalty,
+                   const int32_t *history_ids, const int32_t *history_offsets,
+                   const uint64_t *seeds, uint64_t step,
+                   int32_t *out_tokens, float *out_logprobs,
+                   void *stream, const albireo_sample_ext_t *ext);
+
+/*
+ * The same call with every array in HOST memory (pinned memory makes the copies
+ * asynchronous): copies the inputs to staging space in the workspace, samples, copies
+ * out_tokens / out_logprobs (and the optional ext outputs) back and waits for `stream`.
+ * `history_total` is history_offsets[B] (0 without history).  The pointers inside `ext`
+ * are host pointers too.  Needs the staging bytes in the workspace given to init.
+ */
+int albireo_sample_host(albireo_sampler_t *h,
+                        const void *logits, int32_t B, int32_t V, int32_t dtype,
+                        const float *temperature, const int32_t *top_k,
+                        const float *top_p, const float *min_p,
+                        const float *repetition_penalty, const float *presence_penalty,
+                        const float *frequency_penalty,
+                        const int32_t *history_ids, const int32_t *history_offsets,
+                        int64_t history_total,
+                        const uint64_t *seeds, uint64_t step,
+                        int32_t *out_tokens, float *out_logprobs,
+                        void *stream, const albireo_sample_ext_t *ext);
+
+/* Frees the handle (host memory only). NULL is accepted. */
+int albireo_sample_destroy(albireo_sampler_t *h);
+
+/* Text of the last error recorded on this handle ("" if none); valid until the next call. */
+const char *albireo_last_error(const albireo_sampler_t *h);
+
+/* Number of kernel launches albireo_sample has enqueued through this handle so far. */
+uint64_t albireo_sample_launch_count(const albireo_sampler_t *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALBIREO_SAMPLE_H */

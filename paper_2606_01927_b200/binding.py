@@ -1,0 +1,286 @@
+"""ctypes binding of ``libalbireo_sample.so`` -- argument marshalling only.
+
+Every step of the sampling path runs inside the CUDA library; this module only turns
+torch tensors (device memory, streams) into the pointers and sizes of the C ABI declared
+in ``include/albireo_sample.h``.  There is no CPU fallback: if the library is missing or
+does not load, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import _build
+
+F32 = 0
+BF16 = 1
+OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED = 0, -1, -2, -3, -4
+ROW_GENERAL_PATH, ROW_BAD_PARAM, ROW_HISTORY_OVERFLOW = 1, 2, 4
+FLAG_FORCE_GENERAL = 1
+MAX_VOCAB = 524288
+MAX_NUM_TOP = 128
+
+EXPORTS = [
+    "albireo_sample_workspace_bytes", "albireo_sample_host_staging_bytes", "albireo_sample_init",
+    "albireo_sample", "albireo_sample_host", "albireo_sample_destroy", "albireo_last_error",
+    "albireo_sample_launch_count",
+]
+
+
+class SampleExt(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("flags", C.c_uint32), ("row_stride_elems", C.c_int64),
+        ("row_base", C.c_uint32), ("num_top", C.c_int32),
+        ("out_top_ids", C.c_void_p), ("out_top_logprobs", C.c_void_p),
+        ("out_num_kept", C.c_void_p), ("out_num_topk", C.c_void_p),
+        ("dbg_cap", C.c_int32), ("dbg_topk_ids", C.c_void_p), ("out_row_status", C.c_void_p),
+    ]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+            "(nvcc, sm_100a). The sampler has no CPU fallback.")
+    lib = C.CDLL(path)
+    for name in EXPORTS:
+        if not hasattr(lib, name):
+            raise ImportError(f"{path} does not export {name}")
+    vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+    lib.albireo_sample_workspace_bytes.restype = C.c_size_t
+    lib.albireo_sample_workspace_bytes.argtypes = [i32, i32, i64]
+    lib.albireo_sample_host_staging_bytes.restype = C.c_size_t
+    lib.albireo_sample_host_staging_bytes.argtypes = [i32, i32, i64]
+    lib.albireo_sample_init.restype = C.c_int
+    lib.albireo_sample_init.argtypes = [C.POINTER(vp), i32, i32, i32, i64, vp, C.c_size_t]
+    sample_args = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, u64, vp, vp, vp, C.POINTER(SampleExt)]
+    lib.albireo_sample.restype = C.c_int
+    lib.albireo_sample.argtypes = sample_args
+    lib.albireo_sample_host.restype = C.c_int
+    lib.albireo_sample_host.argtypes = sample_args[:14] + [i64] + sample_args[14:]
+    lib.albireo_sample_destroy.restype = C.c_int
+    lib.albireo_sample_destroy.argtypes = [vp]
+    lib.albireo_last_error.restype = C.c_char_p
+    lib.albireo_last_error.argtypes = [vp]
+    lib.albireo_sample_launch_count.restype = C.c_uint64
+    lib.albireo_sample_launch_count.argtypes = [vp]
+    return lib
+
+
+LIB = _load()
+
+
+class AlbireoError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"albireo_sample error {code}: {msg}")
+        self.code = code
+
+
+def albireo_sample_workspace_bytes(max_rows: int, max_vocab: int, max_history_total: int) -> int:
+    return int(LIB.albireo_sample_workspace_bytes(max_rows, max_vocab, max_history_total))
+
+
+def albireo_sample_host_staging_bytes(max_rows: int, max_vocab: int, max_history_total: int) -> int:
+    return int(LIB.albireo_sample_host_staging_bytes(max_rows, max_vocab, max_history_total))
+
+
+def _dp(t: Optional[torch.Tensor], dtype, device_type: str):
+    if t is None:
+        return None
+    if t.dtype != dtype or not t.is_contiguous() or t.device.type != device_type:
+        raise ValueError(f"expected contiguous {dtype} tensor on {device_type}, got {t.dtype} on {t.device}")
+    return C.c_void_p(t.data_ptr())
+
+
+@dataclass
+class SampleOutputs:
+    tokens: torch.Tensor
+    logprobs: torch.Tensor
+    top_ids: Optional[torch.Tensor] = None
+    top_logprobs: Optional[torch.Tensor] = None
+    num_kept: Optional[torch.Tensor] = None
+    num_topk: Optional[torch.Tensor] = None
+    dbg_topk_ids: Optional[torch.Tensor] = None
+    row_status: Optional[torch.Tensor] = None
+
+
+class Sampler:
+    """Owns a handle from ``albireo_sample_init`` and the torch-allocated workspace."""
+
+    def __init__(self, max_rows: int, max_vocab: int, max_history_total: int = 0,
+                 device: Optional[torch.device] = None, host_staging: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("albireo sampler needs a CUDA device; there is no CPU path")
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.max_rows, self.max_vocab, self.max_history_total = max_rows, max_vocab, max_history_total
+        nbytes = albireo_sample_workspace_bytes(max_rows, max_vocab, max_history_total)
+        if host_staging:
+            nbytes += albireo_sample_host_staging_bytes(max_rows, max_vocab, max_history_total)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 255) & ~255
+        self._handle = C.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = LIB.albireo_sample_init(C.byref(self._handle), self.device.index, max_rows, max_vocab,
+                                         max_history_total, C.c_void_p(self._ws_ptr), nbytes)
+        if rc != OK:
+            raise AlbireoError(rc, "albireo_sample_init failed")
+
+    # -- raw pass-through ------------------------------------------------------------
+    def last_error(self) -> str:
+        return LIB.albireo_last_error(self._handle).decode()
+
+    def launch_count(self) -> int:
+        return int(LIB.albireo_sample_launch_count(self._handle))
+
+    def close(self):
+        if getattr(self, "_handle", None) is not None and self._handle:
+            LIB.albireo_sample_destroy(self._handle)
+            self._handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _ext(self, B, dev_type, device, *, row_base=0, row_stride=0, num_top=0, want_counts=False,
+             dbg_cap=0, want_status=False, flags=0):
+        ext = SampleExt()
+        ext.struct_size = C.sizeof(SampleExt)
+        ext.flags = flags
+        ext.row_stride_elems = row_stride
+        ext.row_base = row_base
+        ext.num_top = num_top
+        out = {}
+        kw = dict(device=device) if dev_type == "cuda" else dict(pin_memory=True)
+        if num_top > 0:
+            out["top_ids"] = torch.empty((B, num_top), dtype=torch.int32, **kw)
+            out["top_logprobs"] = torch.empty((B, num_top), dtype=torch.float32, **kw)
+            ext.out_top_ids = out["top_ids"].data_ptr()
+            ext.out_top_logprobs = out["top_logprobs"].data_ptr()
+        if want_counts:
+            out["num_kept"] = torch.empty(B, dtype=torch.int32, **kw)
+            out["num_topk"] = torch.empty(B, dtype=torch.int32, **kw)
+            ext.out_num_kept = out["num_kept"].data_ptr()
+            ext.out_num_topk = out["num_topk"].data_ptr()
+        if dbg_cap > 0:
+            out["dbg_topk_ids"] = torch.empty((B, dbg_cap), dtype=torch.int32, **kw)
+            ext.dbg_cap = dbg_cap
+            ext.dbg_topk_ids = out["dbg_topk_ids"].data_ptr()
+        if want_status:
+            out["row_status"] = torch.empty(B, dtype=torch.int32, **kw)
+            ext.out_row_status = out["row_status"].data_ptr()
+        return ext, out
+
+    def albireo_sample(self, logits: torch.Tensor, *, temperature=None, top_k=None, top_p=None, min_p=None,
+                       repetition_penalty=None, presence_penalty=None, frequency_penalty=None,
+                       history_ids=None, history_offsets=None, seeds=None, step: int = 0,
+                       out_tokens=None, out_logprobs=None, stream: Optional[torch.cuda.Stream] = None,
+                       row_base: int = 0, num_top: int = 0, want_counts=False, dbg_cap: int = 0,
+                       want_status=False, flags: int = 0, B: Optional[int] = None, V: Optional[int] = None) -> SampleOutputs:
+        """Device-resident call: all tensors on ``self.device``; asynchronous on ``stream``."""
+        if logits.dim() != 2 or logits.stride(1) != 1:
+            raise ValueError("logits must be [B, V] with unit stride along V")
+        B = logits.shape[0] if B is None else B
+        V = logits.shape[1] if V is None else V
+        if logits.dtype == torch.float32:
+            dt = F32
+        elif logits.dtype == torch.bfloat16:
+            dt = BF16
+        else:
+            raise ValueError("logits must be float32 or bfloat16")
+        dev = logits.device
+        if out_tokens is None:
+            out_tokens = torch.empty(B, dtype=torch.int32, device=dev)
+        if out_logprobs is None:
+            out_logprobs = torch.empty(B, dtype=torch.float32, device=dev)
+        row_stride = logits.stride(0) if B > 1 else V
+        ext, extra = self._ext(B, "cuda", dev, row_base=row_base, row_stride=0 if row_stride == V else row_stride,
+                               num_top=num_top, want_counts=want_counts, dbg_cap=dbg_cap,
+                               want_status=want_status, flags=flags)
+        st = torch.cuda.current_stream(dev) if stream is None else stream
+        f32, i32 = torch.float32, torch.int32
+        with torch.cuda.device(dev):
+            rc = LIB.albireo_sample(
+                self._handle, C.c_void_p(logits.data_ptr()), B, V, dt,
+                _dp(temperature, f32, "cuda"), _dp(top_k, i32, "cuda"), _dp(top_p, f32, "cuda"), _dp(min_p, f32, "cuda"),
+                _dp(repetition_penalty, f32, "cuda"), _dp(presence_penalty, f32, "cuda"),
+                _dp(frequency_penalty, f32, "cuda"), _dp(history_ids, i32, "cuda"), _dp(history_offsets, i32, "cuda"),
+                _dp(seeds, torch.int64, "cuda"), C.c_uint64(step),
+                C.c_void_p(out_tokens.data_ptr()), C.c_void_p(out_logprobs.data_ptr()),
+                C.c_void_p(st.cuda_stream), C.byref(ext))
+        if rc != OK:
+            raise AlbireoError(rc, self.last_error())
+        return SampleOutputs(out_tokens, out_logprobs, **extra)
+
+    def albireo_sample_host(self, logits: torch.Tensor, *, temperature=None, top_k=None, top_p=None, min_p=None,
+                            repetition_penalty=None, presence_penalty=None, frequency_penalty=None,
+                            history_ids=None, history_offsets=None, seeds=None, step: int = 0,
+                            out_tokens=None, out_logprobs=None, stream: Optional[torch.cuda.Stream] = None,
+                            row_base: int = 0, num_top: int = 0, want_counts=False, want_status=False,
+                            flags: int = 0) -> SampleOutputs:
+        """Host-buffer call (CPU tensors, ideally pinned): copies in, samples, copies out, waits."""
+        B, V = logits.shape
+        dt = F32 if logits.dtype == torch.float32 else BF16
+        if logits.dtype not in (torch.float32, torch.bfloat16):
+            raise ValueError("logits must be float32 or bfloat16")
+        if out_tokens is None:
+            out_tokens = torch.empty(B, dtype=torch.int32, pin_memory=True)
+        if out_logprobs is None:
+            out_logprobs = torch.empty(B, dtype=torch.float32, pin_memory=True)
+        ext, extra = self._ext(B, "cpu", None, row_base=row_base, num_top=num_top, want_counts=want_counts,
+                               want_status=want_status, flags=flags)
+        st = torch.cuda.current_stream(self.device) if stream is None else stream
+        f32, i32 = torch.float32, torch.int32
+        htot = int(history_ids.numel()) if history_ids is not None else 0
+        with torch.cuda.device(self.device):
+            rc = LIB.albireo_sample_host(
+                self._handle, C.c_void_p(logits.data_ptr()), B, V, dt,
+                _dp(temperature, f32, "cpu"), _dp(top_k, i32, "cpu"), _dp(top_p, f32, "cpu"), _dp(min_p, f32, "cpu"),
+                _dp(repetition_penalty, f32, "cpu"), _dp(presence_penalty, f32, "cpu"),
+                _dp(frequency_penalty, f32, "cpu"), _dp(history_ids, i32, "cpu"), _dp(history_offsets, i32, "cpu"),
+                C.c_int64(htot), _dp(seeds, torch.int64, "cpu"), C.c_uint64(step),
+                C.c_void_p(out_tokens.data_ptr()), C.c_void_p(out_logprobs.data_ptr()),
+                C.c_void_p(st.cuda_stream), C.byref(ext))
+        if rc != OK:
+            raise AlbireoError(rc, self.last_error())
+        return SampleOutputs(out_tokens, out_logprobs, **extra)
+
+
+# ------------------------------------------------------------------ workload marshalling
+
+def workload_tensors(w, device, pinned: bool = False) -> dict:
+    """Moves a ``workloads.Workload`` (numpy) into torch tensors on ``device`` ('cpu' keeps
+    them on the host, pinned if asked).  Pure data movement; seeds travel as the int64
+    view of their uint64 bit patterns."""
+    import numpy as np
+
+    def conv(a, view=None):
+        if a is None:
+            return None
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        if view is not None:
+            t = t.view(view)
+        if str(device) == "cpu":
+            return t.pin_memory() if pinned else t
+        return t.to(device)
+
+    hid = w.history_ids
+    if hid is not None and hid.size == 0:
+        hid = np.zeros(1, dtype=np.int32)      # an empty CSR still needs a non-NULL pointer
+    if w.dtype == F32:
+        logits = conv(w.logits)
+    else:
+        logits = conv(w.logits.view(np.int16), torch.bfloat16)
+    return dict(
+        logits=logits, temperature=conv(w.temperature), top_k=conv(w.top_k), top_p=conv(w.top_p),
+        min_p=conv(w.min_p), repetition_penalty=conv(w.repetition_penalty),
+        presence_penalty=conv(w.presence_penalty), frequency_penalty=conv(w.frequency_penalty),
+        history_ids=conv(hid), history_offsets=conv(w.history_offsets),
+        seeds=conv(None if w.seeds is None else w.seeds.view(np.int64)), step=int(w.step))

@@ -1,0 +1,244 @@
+"""Parity of the CUDA sampler (through the C ABI) with the CPU oracle."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import albireo_oracle as O
+from paper_2606_01927_b200 import workloads as W
+
+from parity import EXCUSED_FRACTION, LOGPROB_TOL, compare, compare_top_lists, to_host
+
+pytestmark = pytest.mark.gpu
+
+DBG_CAP = 128
+_CORES = len(os.sched_getaffinity(0))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2606_01927_b200 import binding as Bd
+    return Bd
+
+
+@pytest.fixture(scope="module")
+def sampler(binding):
+    s = binding.Sampler(max_rows=1024, max_vocab=152064 + 64, max_history_total=1 << 22, host_staging=False)
+    yield s
+    s.close()
+
+
+def run_gpu(binding, sampler, w, *, flags=0, dbg_cap=DBG_CAP):
+    t = binding.workload_tensors(w, sampler.device)
+    out = sampler.albireo_sample(t.pop("logits"), **t, row_base=w.row_base, num_top=w.num_top,
+                                 want_counts=True, dbg_cap=dbg_cap, want_status=True, flags=flags)
+    torch.cuda.synchronize()
+    return to_host(out)
+
+
+def check(binding, sampler, w, *, flags=0, oracle_out=None, allow_excused=None):
+    if oracle_out is None:
+        oracle_out = O.sample(w, threads=_CORES, topk_cap=DBG_CAP)
+    g = run_gpu(binding, sampler, w, flags=flags)
+    rep = compare(w, g, oracle_out, dbg_cap=DBG_CAP)
+    print(rep.summary())
+    assert rep.ok(), rep.failures[:5]
+    limit = math.floor(EXCUSED_FRACTION * w.B) if allow_excused is None else allow_excused
+    assert len(rep.excused) <= limit, rep.excused[:5]
+    bad = compare_top_lists(w, g, oracle_out)
+    assert not bad, bad[:3]
+    return rep, g
+
+
+# ------------------------------------------------------------------ small cases, element by element
+
+SMALL = [
+    # seed, B, V, dtype, quantise
+    (101, 48, 1000, W.F32, None),
+    (102, 48, 1000, W.BF16, None),
+    (103, 40, 4099, W.BF16, None),      # V not a multiple of 8: misaligned rows, scalar head and tail
+    (104, 40, 4099, W.F32, None),
+    (105, 32, 9001, W.BF16, 0.5),       # heavy exact ties at every cut
+    (106, 32, 9001, W.F32, 0.5),
+    (107, 16, 70001, W.BF16, None),     # several tiles per row and a ragged tail
+    (108, 64, 17, W.F32, None),         # V smaller than a warp
+    (109, 1, 33000, W.BF16, None),      # B = 1
+]
+
+
+@pytest.mark.parametrize("seed,B,V,dtype,q", SMALL)
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_small_mixed_parameters(binding, sampler, seed, B, V, dtype, q, flags):
+    w = W.random_small(seed, B=B, V=V, dtype=dtype, quantise=q)
+    w.num_top = 5
+    check(binding, sampler, w, flags=flags, allow_excused=1)
+
+
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_small_no_history_no_arrays(binding, sampler, flags):
+    """All optional arrays NULL: plain softmax sampling over the full row."""
+    rng = np.random.default_rng(5)
+    x = (rng.standard_normal((24, 5000)) * 2).astype(np.float32)
+    w = W.Workload("plain", 24, 5000, W.BF16, W.f32_to_bf16_bits(x))
+    check(binding, sampler, w, flags=flags, allow_excused=1)
+
+
+# ------------------------------------------------------------------ degenerate rows
+
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+def test_degenerate_rows(binding, sampler, dtype, flags):
+    V = 20000
+    rng = np.random.default_rng(17)
+    rows = []
+    rows.append(np.full(V, 1.5, np.float32))                                   # all equal
+    r = np.full(V, -np.inf, np.float32); r[[5, 77, 19999]] = [1.0, 1.0, 0.5]  # fewer finite than k
+    rows.append(r)
+    r = (rng.standard_normal(V) * 0.01).astype(np.float32)                     # near flat
+    rows.append(r)
+    r = (rng.standard_normal(V)).astype(np.float32); r[1234] += 30             # one-hot like
+    rows.append(r)
+    r = np.round(rng.standard_normal(V) * 2).astype(np.float32)                # thousands of ties at the k-th value
+    rows.append(r)
+    r = np.sort((rng.standard_normal(V) * 3).astype(np.float32))               # ascending: worst case for a streaming filter
+    rows.append(r)
+    rows.append(np.sort((rng.standard_normal(V) * 3).astype(np.float32))[::-1].copy())   # descending
+    r = np.zeros(V, np.float32); r[::2] = -0.0                                 # signed zeros
+    rows.append(r)
+    x = np.stack(rows)
+    n = x.shape[0]
+    variants = [
+        dict(temperature=np.full(n, 0.8, np.float32), top_k=np.full(n, 50, np.int32)),
+        dict(temperature=np.full(n, 1.0, np.float32), top_k=np.full(n, 40, np.int32), top_p=np.full(n, 0.9, np.float32)),
+        dict(temperature=np.full(n, 1.0, np.float32), min_p=np.full(n, 0.05, np.float32), top_p=np.full(n, 0.95, np.float32)),
+        dict(temperature=np.full(n, 0.7, np.float32), top_p=np.full(n, 0.5, np.float32)),
+        dict(temperature=np.zeros(n, np.float32)),
+        dict(temperature=np.full(n, 1.3, np.float32), top_k=np.full(n, 1, np.int32)),
+        dict(temperature=np.full(n, 1.0, np.float32), top_k=np.full(n, 300, np.int32), min_p=np.full(n, 1.5, np.float32)),
+        dict(temperature=np.full(n, 1.0, np.float32), top_p=np.zeros(n, np.float32)),
+    ]
+    for i, kw in enumerate(variants):
+        w = W.Workload(f"degenerate{i}", n, V, dtype, x if dtype == W.F32 else W.f32_to_bf16_bits(x),
+                       seeds=np.arange(n, dtype=np.uint64) + 11, step=3, num_top=8, **kw)
+        check(binding, sampler, w, flags=flags, allow_excused=1)
+
+
+def test_history_with_many_distinct_ids_uses_workspace(binding, sampler):
+    """More distinct history ids than the on-chip table holds: counts go through the workspace."""
+    V, B = 30000, 6
+    rng = np.random.default_rng(23)
+    x = (rng.standard_normal((B, V)) * 2).astype(np.float32)
+    lens = np.array([0, 9000, 20000, 5000, 12000, 1], dtype=np.int64)
+    off = np.zeros(B + 1, dtype=np.int64); off[1:] = np.cumsum(lens)
+    ids = rng.integers(0, V, size=int(off[-1])).astype(np.int32)
+    w = W.Workload("manyids", B, V, W.BF16, W.f32_to_bf16_bits(x),
+                   temperature=np.full(B, 0.9, np.float32), top_k=np.full(B, 64, np.int32),
+                   repetition_penalty=np.full(B, 1.2, np.float32), presence_penalty=np.full(B, 0.4, np.float32),
+                   frequency_penalty=np.full(B, 0.1, np.float32),
+                   history_ids=ids, history_offsets=off.astype(np.int32), seeds=np.arange(B, dtype=np.uint64))
+    for flags in (0, 1):
+        rep, g = check(binding, sampler, w, flags=flags, allow_excused=0)
+        assert not (g["row_status"] & binding.ROW_HISTORY_OVERFLOW).any()
+
+
+# ------------------------------------------------------------------ the five configurations and the metric workload
+
+_ORACLE_CACHE = {}
+
+
+def oracle_for(name):
+    if name not in _ORACLE_CACHE:
+        w = W.make(name)
+        _ORACLE_CACHE[name] = (w, O.sample(w, threads=_CORES, topk_cap=DBG_CAP))
+    return _ORACLE_CACHE[name]
+
+
+@pytest.mark.parametrize("name", ["config1", "config2", "configM", "config3", "config4", "config5"])
+def test_config_parity(binding, sampler, name):
+    w, o = oracle_for(name)
+    rep, g = check(binding, sampler, w, oracle_out=o)
+    # greedy rows are bit-exact by construction of compare(); report the path mix
+    print(name, "general-path rows:", rep.general_rows, "of", w.B)
+
+
+@pytest.mark.parametrize("name", ["config1", "config3", "config4"])
+def test_config_parity_general_path(binding, sampler, name):
+    """The same configurations with every row forced down the general path."""
+    w, o = oracle_for(name)
+    check(binding, sampler, w, flags=1, oracle_out=o, allow_excused=max(1, math.floor(EXCUSED_FRACTION * w.B)))
+
+
+# ------------------------------------------------------------------ properties that hold at any size
+
+def test_shard_invariance_and_padding_rows(binding, sampler):
+    w = W.config3(B=24, V=20000, hist_len=300)
+    full = run_gpu(binding, sampler, w)
+    a = run_gpu(binding, sampler, w.rows(0, 10))
+    b = run_gpu(binding, sampler, w.rows(10, 24))
+    assert (np.concatenate([a["tokens"], b["tokens"]]) == full["tokens"]).all()
+    assert (np.concatenate([a["logprobs"], b["logprobs"]]).view(np.uint32) == full["logprobs"].view(np.uint32)).all()
+
+
+def test_repeated_launches_are_bit_identical(binding, sampler):
+    w = W.config4(B=64, V=50000, max_hist=1000)
+    a = run_gpu(binding, sampler, w)
+    for _ in range(3):
+        b = run_gpu(binding, sampler, w)
+        for k in ("tokens", "num_kept", "num_topk"):
+            assert (a[k] == b[k]).all()
+        assert (a["logprobs"].view(np.uint32) == b["logprobs"].view(np.uint32)).all()
+
+
+def test_row_stride_and_stream(binding, sampler):
+    """Rows taken out of a wider buffer (row stride > V) on a side stream."""
+    w = W.config1(B=8, V=3000)
+    t = binding.workload_tensors(w, sampler.device)
+    wide = torch.zeros((8, 3000 + 40), dtype=torch.float32, device=sampler.device)
+    wide[:, :3000] = t["logits"]
+    view = wide[:, :3000]
+    st = torch.cuda.Stream(device=sampler.device)
+    st.wait_stream(torch.cuda.current_stream())
+    t.pop("logits")
+    with torch.cuda.stream(st):
+        out = sampler.albireo_sample(view, **t, stream=st, want_counts=True)
+    st.synchronize()
+    ref = run_gpu(binding, sampler, w)
+    assert (out.tokens.cpu().numpy() == ref["tokens"]).all()
+    assert (out.logprobs.cpu().numpy() == ref["logprobs"]).all()
+
+
+def test_host_entry_matches_device_entry(binding):
+    w = W.config3(B=16, V=20000, hist_len=500)
+    w.num_top = 4
+    s = binding.Sampler(max_rows=16, max_vocab=20000, max_history_total=16 * 500, host_staging=True)
+    t = binding.workload_tensors(w, "cpu", pinned=True)
+    h = s.albireo_sample_host(t.pop("logits"), **t, num_top=4, want_counts=True, want_status=True)
+    td = binding.workload_tensors(w, s.device)
+    d = s.albireo_sample(td.pop("logits"), **td, num_top=4, want_counts=True, want_status=True)
+    torch.cuda.synchronize()
+    assert (h.tokens.numpy() == d.tokens.cpu().numpy()).all()
+    assert (h.logprobs.numpy() == d.logprobs.cpu().numpy()).all()
+    assert (h.top_ids.numpy() == d.top_ids.cpu().numpy()).all()
+    assert (h.num_kept.numpy() == d.num_kept.cpu().numpy()).all()
+    o = O.sample(w, threads=_CORES)
+    assert (h.tokens.numpy() == o.tokens).all()
+    s.close()
+
+
+def test_argument_errors_launch_nothing(binding, sampler):
+    x = torch.zeros((4, 100), dtype=torch.float32, device=sampler.device)
+    n0 = sampler.launch_count()
+    with pytest.raises(binding.AlbireoError) as e:
+        sampler.albireo_sample(x, B=2000)
+    assert e.value.code == binding.EINVAL
+    with pytest.raises(binding.AlbireoError):
+        sampler.albireo_sample(x, num_top=binding.MAX_NUM_TOP + 1)
+    with pytest.raises(binding.AlbireoError):
+        sampler.albireo_sample(x, history_offsets=torch.zeros(5, dtype=torch.int32, device=sampler.device))
+    out = sampler.albireo_sample(x, B=0)
+    assert sampler.launch_count() == n0
+    sampler.albireo_sample(x)
+    torch.cuda.synchronize()
+    assert sampler.launch_count() == n0 + 1
