@@ -1,0 +1,337 @@
+#!/usr/bin/env python
+"""Benchmark of the batched token sampler: rows sampled per second and the fraction of
+the HBM roofline on the metric workload (B=256 rows, V=152064, bf16, top-k + top-p).
+
+A "step" is one pass of the whole sampling path over one batch: one `albireo_sample`
+call (penalties -> temperature -> top-k -> min-p/top-p -> softmax/logprob -> race).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+N > 1 (launched by torch.distributed.run, one rank per GPU): rows are independent
+(section 6.1 of the paper), so every rank samples its own B rows with global row ids
+`rank * B + b` and there is no data-path collective ("weak" scaling).
+
+`--impl reference` times the CPU oracle instead (rank 0 only), each step a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "rows_sampled_per_s"
+UNIT = "rows/s"
+N_ROTATING = 8            # distinct logits buffers, so that no call finds its rows in L2
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of albireo_sample_kernel on the
+# metric workload, from the ncu capture summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"configM": None}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.stop = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception as e:   # NVML missing: report that, do not guess
+            self.err = repr(e)
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), mhz, int(reasons)))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.ok:
+            self.thread.start()
+
+    def finish(self, t0: float, t1: float):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable"]}
+        self.stop.set()
+        self.thread.join(timeout=2)
+        nv = self.nv
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        used = inside if len(inside) >= 3 else self.samples
+        names = {
+            "gpu_idle": 0x1, "applications_clocks_setting": 0x2, "sw_power_cap": 0x4, "hw_slowdown": 0x8,
+            "sync_boost": 0x10, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+            "hw_power_brake_slowdown": 0x80, "display_clock_setting": 0x100,
+        }
+        bits = 0
+        for s in used:
+            bits |= s[2]
+        reasons = sorted(n for n, m in names.items() if bits & m and n != "gpu_idle")
+        return {"sm_mhz": statistics.median(s[1] for s in used) if used else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples_in_timed_region": len(inside), "samples_total": len(self.samples)}
+
+
+def describe(w) -> str:
+    def one(a, fmt):
+        if a is None:
+            return "off"
+        return fmt % a[0] if np.all(a == a[0]) else "per-row"
+    return (f"{w.name}: B={w.B} V={w.V} {'bf16' if w.dtype == 1 else 'f32'} T={one(w.temperature, '%.2g')} "
+            f"top_k={one(w.top_k, '%d')} top_p={one(w.top_p, '%.2g')} min_p={one(w.min_p, '%.2g')} "
+            f"history={'none' if w.history_ids is None else str(int(w.history_ids.size)) + ' ids'}")
+
+
+def algorithmic_bytes(w) -> int:
+    """Bytes one launch must move: every logit once, the history CSR, per-row scalars, outputs."""
+    n_param_arrays = sum(a is not None for a in (w.temperature, w.top_k, w.top_p, w.min_p, w.repetition_penalty,
+                                                 w.presence_penalty, w.frequency_penalty))
+    return w.logit_bytes + w.history_bytes + w.B * (4 * n_param_arrays + 8 + 8)
+
+
+def run_reference(args, w):
+    """The CPU oracle as it stands, on the host cores, on a bounded sample of the workload."""
+    from oracle import albireo_oracle as O
+    cores = len(os.sched_getaffinity(0))
+    rows = min(w.B, max(cores, args.ref_rows))
+    sub = w.rows(0, rows)
+    for _ in range(min(args.warmup, 1)):
+        O.sample(sub, threads=cores)
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        O.sample(sub, threads=cores)
+        times.append(time.perf_counter() - t0)
+    per_step = sum(times) / len(times)
+    value = rows / per_step
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": per_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(w), "sample": f"first {rows} rows of the batch per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {rows} of {w.B} rows per step, {args.steps} steps, one thread per core"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="albireo", choices=["albireo", "reference"])
+    ap.add_argument("--workload", default="configM")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--ref-rows", type=int, default=64, help="rows per step of the reference arm")
+    ap.add_argument("--no-graph", action="store_true", help="launch each step from Python instead of one CUDA graph")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--general-path", action="store_true", help="force every row down the general path")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2606_01927_b200 import workloads as W
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, W.make(args.workload))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2606_01927_b200 import _build
+    _build.build()
+    from paper_2606_01927_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the sampler has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = W.make(args.workload)
+    w.row_base = rank * w.B                      # global row ids: draws do not depend on the sharding
+    htot = 0 if w.history_ids is None else int(w.history_ids.size)
+    sampler = binding.Sampler(max_rows=w.B, max_vocab=w.V, max_history_total=htot, device=dev, host_staging=True)
+    t = binding.workload_tensors(w, dev)
+    logits0 = t.pop("logits")
+    # rotating copies (rows rolled so the copies are not byte-identical)
+    bufs = [logits0] + [torch.roll(logits0, shifts=i, dims=0).contiguous() for i in range(1, N_ROTATING)]
+    out_tok = torch.empty(w.B, dtype=torch.int32, device=dev)
+    out_lp = torch.empty(w.B, dtype=torch.float32, device=dev)
+    flags = binding.FLAG_FORCE_GENERAL if args.general_path else 0
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(i, st):
+        sampler.albireo_sample(bufs[i % N_ROTATING], **t, out_tokens=out_tok, out_logprobs=out_lp, stream=st,
+                               row_base=w.row_base, flags=flags)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    clocks = ClockSampler(local_rank)
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            step(i, stream)
+    torch.cuda.synchronize(dev)
+
+    graph = None
+    if not args.no_graph:
+        # the K launches of the timed region as one CUDA graph: the region is launch-bound otherwise
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(args.steps):
+                step(i, stream)
+        graph.replay()                              # one untimed replay (uploads the graph)
+        torch.cuda.synchronize(dev)
+
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    clocks.start()
+    n_before = sampler.launch_count()
+    barrier()
+    t_wall0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        if graph is not None:
+            graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i, stream)
+        e1.record(stream)
+    barrier()
+    t_wall1 = time.perf_counter()
+    # under graph replay the launches were counted at capture time
+    launches = args.steps if graph is not None else sampler.launch_count() - n_before
+    elapsed_ms = e0.elapsed_time(e1)
+    clock_info = clocks.finish(t_wall0, t_wall1)
+
+    # isolated launches, each bracketed by its own events (context for the roofline)
+    iso = []
+    with torch.cuda.stream(stream):
+        for i in range(min(args.steps, 50)):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            step(i, stream)
+            b.record(stream)
+            iso.append((a, b))
+    torch.cuda.synchronize(dev)
+    iso_us = statistics.median(a.elapsed_time(b) for a, b in iso) * 1e3
+
+    if world > 1:
+        tt = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * w.B / (ms_per_step * 1e-3)
+
+    # end to end: host buffers through the C-ABI host entry, copies inside the timed region
+    th = binding.workload_tensors(w, "cpu", pinned=True)
+    h_logits = th.pop("logits")
+    h_tok = torch.empty(w.B, dtype=torch.int32, pin_memory=True)
+    h_lp = torch.empty(w.B, dtype=torch.float32, pin_memory=True)
+    h2d = sum(int(v.numel() * v.element_size()) for v in [h_logits] + [x for x in th.values() if torch.is_tensor(x)])
+    d2h = int(h_tok.numel() * 4 + h_lp.numel() * 4)
+
+    def e2e_step():
+        sampler.albireo_sample_host(h_logits, **th, out_tokens=h_tok, out_logprobs=h_lp, stream=stream,
+                                    row_base=w.row_base, flags=flags)
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize(dev)
+    e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+    if world > 1:
+        tt = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_s = float(tt.item())
+    e2e_value = world * w.B / e2e_s
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        alg = algorithmic_bytes(w)
+        achieved = alg / (ms_per_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": describe(w), "rows_per_gpu": w.B,
+                "l2": f"{N_ROTATING} rotating logits buffers ({N_ROTATING * w.logit_bytes / 1e6:.0f} MB per GPU) so no call finds its rows in the 126 MB L2",
+                "launch": "one CUDA graph of K launches" if graph is not None else "K launches from the host",
+                "path": "general path forced" if args.general_path else "automatic",
+            },
+            "tokens_per_s": value,
+            "roofline": {
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+                "algorithmic_bytes_per_launch": alg, "kernel": "albireo_sample_kernel",
+                "launch_us_avg_timed_region": ms_per_step * 1e3, "launch_us_median_isolated": iso_us,
+                "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
+            },
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps},
+            "gpu_launches": launches,
+            "clocks": clock_info,
+        }
+        if world == 1 and not args.skip_cpu_baseline:
+            from oracle import albireo_oracle as O
+            cores = len(os.sched_getaffinity(0))
+            t0 = time.perf_counter()
+            O.sample(w, threads=cores)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": w.B / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"all {w.B} rows of the batch once, one thread per core ({dt:.2f} s wall)"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -82,8 +82,9 @@ typedef struct albireo_sample_ext {
     int32_t *out_num_topk;     /* [B] device: size of the set kept by the top-k stage       */
     int32_t dbg_cap;           /* capacity per row of dbg_topk_ids                          */
     int32_t *dbg_topk_ids;     /* [B, dbg_cap] device: ids kept by the top-k stage, in no
-                                  particular order, -1 padded; written only for rows whose
-                                  top-k stage keeps <= dbg_cap ids                          */
+                                  particular order, -1 padded; written only for rows with an
+                                  active top-k (1 <= k < V, or greedy) whose top-k stage
+                                  keeps <= dbg_cap ids                                      */
     uint32_t *out_row_status;  /* [B] device: ALBIREO_ROW_* bits                            */
 } albireo_sample_ext_t;
 

@@ -16,6 +16,7 @@
 // the order-preserving map of fp32 bit patterns.  Larger C comes first; all C distinct.
 // A kept set is always a prefix of that order, i.e. { t : C(t) >= threshold }.
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdio.h>
@@ -32,6 +33,11 @@ constexpr int NT = 512;                 // threads per CTA
 constexpr int NWARPS = NT / 32;
 constexpr int HIST_BINS = 2048;         // 11-bit digits
 constexpr int CNT_CAP = 4096;           // on-chip slots for distinct history ids per row
+constexpr int CAND_CAP = 2048;          // candidate buffer entries (candidate path)
+constexpr int SORT_MAX = 512;           // most candidates the final stage sorts (== NT)
+constexpr int KA_MAX = 256;             // largest top-k the candidate path takes
+constexpr int TILE_VECS = 4;            // 16-byte vectors per thread per tile
+constexpr double FX50 = 1125899906842624.0;        // 2^50: fixed-point scale of the final stage
 constexpr uint32_t KEY_MIN_FINITE = 0x00800000u;   // key(-FLT_MAX); key(-inf) is one below
 constexpr uint32_t KEY_POS_INF = 0xFF800000u;      // key(+inf)
 constexpr float FX_SCALE = 1099511627776.0f;       // 2^40: fixed-point scale of masses
@@ -126,6 +132,7 @@ struct BlockScratch {
     uint32_t found_digit, found_cnt;
     u64 found_above;
     uint32_t list_cnt;
+    uint32_t cand_cnt, overflow, runmax;
 };
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -517,7 +524,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         C1 = select_by_count<DT>(s, h, c, Cfin, n_topk, 0, 0);
     }
     out.n_topk = (int32_t)n_topk;
-    if (a.dbg_topk_ids && n_topk <= (u64)a.dbg_cap) {
+    if (a.dbg_topk_ids && rp.top_k >= 1 && rp.top_k < V && n_topk <= (u64)a.dbg_cap) {
         if (threadIdx.x == 0) s.list_cnt = 0;
         __syncthreads();
         int32_t *dst = a.dbg_topk_ids + (int64_t)b * a.dbg_cap;
@@ -583,9 +590,384 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     }
 }
 
+
+// ------------------------------------------------------------------ candidate path
+//
+// One streaming pass over the row.  A conservative threshold tau (an order key) is kept
+// such that every element of the final kept set has key >= tau: the k-th largest key
+// among the candidates seen so far (top-k), and/or the min-p floor below the running
+// maximum.  Elements below tau are dropped by a cheap vector test; the rest are checked
+// exactly and appended to a small on-chip candidate list, which is then sorted and cut.
+// Penalised tokens never enter through the stream (their raw value is not their score):
+// they are evaluated from the history bitmap after the stream.
+
+struct CandSmem {
+    u64 *cand;        // CAND_CAP composites
+    u64 *sorted;      // SORT_MAX composites, best first
+    uint32_t *hist;   // 256 bins
+};
+
+__device__ __forceinline__ void cand_append(BlockScratch &s, u64 *cand, u64 C) {
+    uint32_t slot = atomicAdd(&s.cand_cnt, 1u);
+    if (slot < (uint32_t)CAND_CAP) cand[slot] = C; else s.overflow = 1u;
+    atomicMax(&s.runmax, (uint32_t)(C >> 32));
+}
+
+// k-th largest key (1-based) among cand[0..n), n >= k: 8-bit radix select.  Uniform result.
+__device__ uint32_t cand_select_key(BlockScratch &s, const CandSmem &cs, int n, int k) {
+    uint32_t prefix = 0;
+    uint32_t rank = (uint32_t)k;
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        if (threadIdx.x < 256) cs.hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += NT) {
+            uint32_t key = (uint32_t)(cs.cand[i] >> 32);
+            if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&cs.hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            const int lane = threadIdx.x;
+            uint32_t local = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) local += cs.hist[255 - (lane * 8 + q)];
+            uint32_t inc = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
+            uint32_t run = inc - local;
+            if (run < rank && rank <= run + local) {
+                for (int q = 0; q < 8; ++q) {
+                    uint32_t v = cs.hist[255 - (lane * 8 + q)];
+                    if (rank <= run + v) { s.found_digit = 255 - (lane * 8 + q); s.found_above = run; break; }
+                    run += v;
+                }
+            }
+        }
+        __syncthreads();
+        rank -= (uint32_t)s.found_above;
+        prefix = (prefix << 8) | s.found_digit;
+    }
+    return prefix;
+}
+
+// keeps the candidates with key >= tkey; returns the new count (uniform)
+__device__ int cand_compact(BlockScratch &s, const CandSmem &cs, int n, uint32_t tkey) {
+    constexpr int PER = CAND_CAP / NT;
+    u64 mine[PER];
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        int i = threadIdx.x + q * NT;
+        mine[q] = (i < n) ? cs.cand[i] : 0ull;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) s.cand_cnt = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < PER; ++q) {
+        if ((uint32_t)(mine[q] >> 32) >= tkey && mine[q] != 0ull) {
+            uint32_t slot = atomicAdd(&s.cand_cnt, 1u);
+            cs.cand[slot] = mine[q];
+        }
+    }
+    __syncthreads();
+    return (int)s.cand_cnt;
+}
+
+// Vector pre-test per dtype.  RawThr is the threshold in the domain the test runs in:
+// bf16: the smallest raw bf16 whose score has key >= tau (packed twice); fp32: unkey(tau).
+template <int DT> struct VecTest;
+template <> struct VecTest<ALBIREO_BF16> {
+    static __device__ uint32_t raw_threshold(uint32_t tau_key, float invT) {
+        const float tz = unkey(tau_key);
+        const float xg = __fdiv_rn(tz, invT);
+        const uint32_t b16 = __float_as_uint(xg) >> 16;
+        uint32_t k16 = (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
+        auto bits_of = [](uint32_t kk) { return (kk & 0x8000u) ? (kk & 0x7FFFu) : (~kk & 0xFFFFu); };
+        auto passes = [&](uint32_t kk) {
+            float x = __uint_as_float(bits_of(kk) << 16);
+            return key_of(__fmul_rn(x, invT)) >= tau_key;
+        };
+        if (k16 < 0x0080u) k16 = 0x0080u;
+        if (k16 > 0xFF7Fu) k16 = 0xFF7Fu;
+        int it = 0;
+        while (it < 16 && k16 > 0x0080u && passes(k16)) { --k16; ++it; }
+        while (it < 32 && k16 < 0xFF7Fu && !passes(k16)) { ++k16; ++it; }
+        const bool ok = passes(k16) && (k16 == 0x0080u || !passes(k16 - 1));
+        const uint32_t b = ok ? bits_of(k16) : 0xFF80u;     // not settled: let everything through
+        return b | (b << 16);
+    }
+    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
+        __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x), *reinterpret_cast<const __nv_bfloat162 *>(&q.y));
+        __nv_bfloat162 b2 = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&q.z), *reinterpret_cast<const __nv_bfloat162 *>(&q.w));
+        a = __hmax2(a, b2);
+        return __hge2_mask(a, *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
+    }
+    static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
+};
+template <> struct VecTest<ALBIREO_F32> {
+    static __device__ uint32_t raw_threshold(uint32_t tau_key, float) { return __float_as_uint(unkey(tau_key)); }
+    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float invT) {
+        float m = fmaxf(fmaxf(__fmul_rn(__uint_as_float(q.x), invT), __fmul_rn(__uint_as_float(q.y), invT)),
+                        fmaxf(__fmul_rn(__uint_as_float(q.z), invT), __fmul_rn(__uint_as_float(q.w), invT)));
+        return m >= __uint_as_float(thr);
+    }
+    static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
+};
+
+// exact check of one vector's unpenalised elements against tau; appends survivors
+template <int DT>
+__device__ __noinline__ void slow_vector(BlockScratch &s, u64 *cand, const RowCtx &c, uint4 q, int i0,
+                                         uint32_t tau_key, u64 skip) {
+    typedef Elem<DT> E;
+    uint32_t m = 0;
+    if (c.has_hist) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+#pragma unroll
+    for (int e = 0; e < E::PER_VEC; ++e) {
+        if (m & (1u << e)) continue;
+        uint32_t key = key_of(__fmul_rn(E::get(q, e), c.invT));
+        u64 C = comp_of(key, i0 + e);
+        if (key >= tau_key && C != skip) cand_append(s, cand, C);
+    }
+}
+
+// Returns false if the row must be handled by the general path instead.
+template <int DT>
+__device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const RowCtx &c, const RowParams &rp,
+                               const SampleArgs &a, int b, RowOut &out) {
+    typedef Elem<DT> E;
+    typedef VecTest<DT> T;
+    const int V = c.V;
+    const int k = rp.greedy ? 1 : rp.top_k;
+    const bool has_topk = rp.greedy || (k >= 1 && k < V);
+    const bool has_minp = !rp.greedy && rp.min_p > 0.0f;
+    if (has_topk && k > KA_MAX) return false;
+    if (!has_topk && !has_minp) return false;
+    // with the debug id list requested, keep the stream's threshold purely top-k so that the
+    // top-k stage's set is known exactly
+    const bool stream_minp = has_minp && !(has_topk && a.dbg_topk_ids != nullptr);
+    const double ln_minp = has_minp ? log((double)rp.min_p) : 0.0;
+
+    if (threadIdx.x == 0) { s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; }
+    __syncthreads();
+
+    const uintptr_t addr = (uintptr_t)c.row;
+    int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
+    if (head > V) head = V;
+    const int nvec = (V - head) / E::PER_VEC;
+    const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
+    const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
+
+    uint32_t tau_key = KEY_MIN_FINITE;
+    uint32_t thr = T::raw_threshold(tau_key, c.invT);
+    uint32_t seen_max = 0;
+
+    auto floor_from_max = [&](uint32_t maxkey) -> uint32_t {
+        // a key no larger than the key of the smallest score that passes min-p under this maximum
+        return minp_key(unkey(maxkey), rp.min_p);
+    };
+
+    uint4 cur[TILE_VECS], nxt[TILE_VECS];
+#pragma unroll
+    for (int u = 0; u < TILE_VECS; ++u) {
+        int v = u * NT + threadIdx.x;
+        cur[u] = (v < nvec) ? __ldg(vp + v) : T::fill();
+    }
+    for (int tile = 0; tile < ntiles; ++tile) {
+        const int vbase = tile * NT * TILE_VECS;
+        if (tile + 1 < ntiles) {
+#pragma unroll
+            for (int u = 0; u < TILE_VECS; ++u) {
+                int v = vbase + NT * TILE_VECS + u * NT + threadIdx.x;
+                nxt[u] = (v < nvec) ? __ldg(vp + v) : T::fill();
+            }
+        }
+        u64 own = 0;
+        if (tile == 0) {
+            // warm-up: every thread contributes its best unpenalised element; the k-th largest
+            // of these is a valid lower bound of the row's k-th largest score
+#pragma unroll
+            for (int u = 0; u < TILE_VECS; ++u) {
+                const int i0 = head + (vbase + u * NT + threadIdx.x) * E::PER_VEC;
+                uint32_t m = 0;
+                if (c.has_hist && i0 < V) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+#pragma unroll
+                for (int e = 0; e < E::PER_VEC; ++e) {
+                    uint32_t key = key_of(__fmul_rn(E::get(cur[u], e), c.invT));
+                    u64 C = comp_of(key, i0 + e);
+                    if (!(m & (1u << e)) && key >= KEY_MIN_FINITE && C > own) own = C;
+                }
+            }
+            if (own) cand_append(s, cs.cand, own);
+            __syncthreads();
+            int n = (int)s.cand_cnt;
+            uint32_t rmax = s.runmax;
+            __syncthreads();
+            if (has_topk && n >= k) tau_key = cand_select_key(s, cs, n, k);
+            if (stream_minp && rmax) { uint32_t f = floor_from_max(rmax); tau_key = f > tau_key ? f : tau_key; }
+            seen_max = rmax;
+            thr = T::raw_threshold(tau_key, c.invT);
+        }
+#pragma unroll
+        for (int u = 0; u < TILE_VECS; ++u) {
+            const int v = vbase + u * NT + threadIdx.x;
+            if (v < nvec && T::may_pass(cur[u], thr, c.invT))
+                slow_vector<DT>(s, cs.cand, c, cur[u], head + v * E::PER_VEC, tau_key, own);
+        }
+        __syncthreads();                       // every append of this tile is done
+        int n = (int)s.cand_cnt;
+        const uint32_t ovf = s.overflow, rmax = s.runmax;
+        __syncthreads();                       // nobody appends again before all have read
+        if (ovf) return false;
+        bool changed = false;
+        if (has_topk && n >= k && (n >= 2 * k + 32 || n > CAND_CAP / 2 || tile == 0)) {
+            uint32_t t = cand_select_key(s, cs, n, k);
+            if (t > tau_key) { tau_key = t; changed = true; }
+            n = cand_compact(s, cs, n, tau_key);
+        }
+        if (stream_minp && rmax != seen_max) {
+            seen_max = rmax;
+            uint32_t f = floor_from_max(rmax);
+            if (f > tau_key) { tau_key = f; changed = true; }
+        }
+        if (!has_topk && n > CAND_CAP / 2) n = cand_compact(s, cs, n, tau_key);
+        if (changed) thr = T::raw_threshold(tau_key, c.invT);
+#pragma unroll
+        for (int u = 0; u < TILE_VECS; ++u) cur[u] = nxt[u];
+    }
+    // scalar head and tail of a row that is not 16-byte aligned / not a whole number of vectors
+    {
+        const int tail0 = head + nvec * E::PER_VEC;
+        const int nscal = head + (V - tail0);
+        for (int q = threadIdx.x; q < nscal; q += NT) {
+            int i = q < head ? q : tail0 + (q - head);
+            if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
+            uint32_t key = key_of(__fmul_rn(E::load(c.row, i), c.invT));
+            if (key >= tau_key) cand_append(s, cs.cand, comp_of(key, i));
+        }
+    }
+    // penalised tokens, straight from the history bitmap
+    if (c.has_hist) {
+        const int nwords = (V + 31) >> 5;
+        for (int w = threadIdx.x; w < nwords; w += NT) {
+            uint32_t bits = c.bitmap[w];
+            if (!bits) continue;
+            uint32_t r = c.coarse[w >> 3];
+            for (int ww = (w >> 3) << 3; ww < w; ++ww) r += __popc(c.bitmap[ww]);
+            while (bits) {
+                int bit = __ffs(bits) - 1;
+                bits &= bits - 1;
+                int i = (w << 5) + bit;
+                float x = E::load(c.row, i);
+                uint32_t cnt = c.counts[r++];
+                float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
+                av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cnt)));
+                av = __fsub_rn(av, c.p);
+                uint32_t key = key_of(__fmul_rn(av, c.invT));
+                if (key >= tau_key) cand_append(s, cs.cand, comp_of(key, i));
+            }
+        }
+    }
+    __syncthreads();
+    int n = (int)s.cand_cnt;
+    const uint32_t ovf = s.overflow;
+    const uint32_t kmax = s.runmax;
+    __syncthreads();
+    if (ovf || n < 1) return false;
+
+    // exact top-k threshold, then the exact min-p floor for rows without a top-k
+    bool topk_exact_known = true;      // is min(k, #finite) known without counting?
+    if (has_topk) {
+        if (n > k) {
+            uint32_t t = cand_select_key(s, cs, n, k);
+            n = cand_compact(s, cs, n, t);
+        } else if (n < k && stream_minp) {
+            topk_exact_known = false;
+        }
+    } else {
+        n = cand_compact(s, cs, n, floor_from_max(kmax));
+        topk_exact_known = false;
+    }
+    if (n > SORT_MAX || n < 1) return false;
+
+    // sort by rank counting (all composites distinct)
+    if (threadIdx.x < n) {
+        const u64 C = cs.cand[threadIdx.x];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += cs.cand[j] > C;
+        cs.sorted[rank] = C;
+    }
+    __syncthreads();
+
+    const int j = threadIdx.x;
+    const u64 Cj = j < n ? cs.sorted[j] : 0ull;
+    const float zmax = unkey((uint32_t)(cs.sorted[0] >> 32));
+    const float zj = unkey((uint32_t)(Cj >> 32));
+    const double dj = (double)zj - (double)zmax;
+    const int L6 = has_topk ? (n < k ? n : k) : n;
+
+    int n_topk = L6;
+    if (!topk_exact_known && a.out_num_topk) {
+        // diagnostic only: count the finite scores of the row
+        uint32_t local = 0;
+        for_each_score<DT>(c, [&](int, float z) { uint32_t kk = key_of(z); local += (kk >= KEY_MIN_FINITE && kk < KEY_POS_INF); });
+        u64 nfin = block_sum_u64(s, local);
+        n_topk = has_topk ? (int)(nfin < (u64)k ? nfin : (u64)k) : (int)nfin;
+    }
+    out.n_topk = n_topk;
+    if (a.dbg_topk_ids && has_topk && L6 <= a.dbg_cap && j < L6) a.dbg_topk_ids[(int64_t)b * a.dbg_cap + j] = comp_idx(Cj);
+
+    // min-p (a prefix of the order), at least one survivor
+    bool in7 = j < L6 && (!has_minp || dj >= ln_minp);
+    int L7 = (int)block_sum_u64(s, in7 ? 1u : 0u);
+    if (L7 < 1) L7 = 1;
+    // top-p over the survivors' mass, fixed-point so that the sums do not depend on the order
+    u64 ej = (j < L7) ? __double2ull_rn(exp(dj) * FX50) : 0ull;
+    u64 total;
+    u64 before = block_exscan_u64(s, ej, total);
+    bool keep = j < L7;
+    if (!rp.greedy && rp.top_p < 1.0f) {
+        double t = ceil((double)rp.top_p * (double)total);
+        u64 target = t <= 1.0 ? 1ull : (u64)t;
+        if (target > total) target = total;
+        keep = keep && before < target;
+    }
+    const int L8 = (int)block_sum_u64(s, keep ? 1u : 0u);
+    const u64 S_fx = block_sum_u64(s, keep ? ej : 0ull);
+    const double lnS = log((double)S_fx) - 50.0 * 0.6931471805599453;
+    out.n_keep = L8;
+
+    // race
+    const int id = comp_idx(Cj);
+    u64 G = 0;
+    if (keep) {
+        double g = dj + neg_log_exp1_f64(race_word(rp.seed, rp.R, a.step, id));
+        long long gb = __double_as_longlong(g);
+        G = (gb < 0) ? ~(u64)gb : ((u64)gb | 0x8000000000000000ull);
+    }
+    const u64 Gmax = block_max_u64(s, G);
+    const u64 win = block_max_u64(s, (keep && G == Gmax) ? (u64)(uint32_t)(~(uint32_t)id) : 0ull);
+    const int tok = (L8 == 1) ? comp_idx(cs.sorted[0]) : (int)(~(uint32_t)win);
+    if (keep && id == tok) {
+        s.bcast[0] = (u64)__float_as_uint((L8 == 1) ? 0.0f : (float)(dj - lnS));
+    }
+    __syncthreads();
+    out.token = tok;
+    out.logprob = __uint_as_float((uint32_t)s.bcast[0]);
+    if (a.num_top > 0 && j < a.num_top) {
+        const int64_t q = (int64_t)b * a.num_top + j;
+        if (j < L8) {
+            a.out_top_ids[q] = id;
+            a.out_top_logprobs[q] = (L8 == 1) ? 0.0f : (float)(dj - lnS);
+        }
+    }
+    __syncthreads();
+    return true;
+}
+
 // ------------------------------------------------------------------ the kernel
 
-// dynamic shared memory layout (bytes): [hist cnt 8 KiB][hist mass 16 KiB][bitmap][coarse][counts]
+// dynamic shared memory layout (bytes): [24 KiB shared by the two paths: histograms (cnt 8 KiB, mass
+// 16 KiB) or candidates (16 KiB) + sorted list (4 KiB) + 256 bins (1 KiB)][bitmap][coarse][counts]
 template <int DT>
 __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -642,7 +1024,16 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     }
     __syncthreads();
 
-    general_path<DT>(s, h, c, rp, a, b, out);
+    CandSmem cs;
+    cs.cand = (u64 *)smem;                                  // 16 KiB
+    cs.sorted = (u64 *)(smem + CAND_CAP * 8);               // 4 KiB
+    cs.hist = (uint32_t *)(smem + CAND_CAP * 8 + SORT_MAX * 8);   // 1 KiB
+    bool done = false;
+    if (!(a.flags & ALBIREO_FLAG_FORCE_GENERAL)) done = candidate_path<DT>(s, cs, c, rp, a, b, out);
+    if (!done) {
+        __syncthreads();
+        general_path<DT>(s, h, c, rp, a, b, out);
+    }
 
     if (threadIdx.x == 0) {
         a.out_tokens[b] = out.token;

@@ -2,8 +2,9 @@
 
 Rules (tolerances written out here, nowhere else):
   * greedy rows: token bit-exact, logprob exactly 0;
-  * top-k stage: the number of ids kept is equal in every row, and the id set is
-    bit-exact wherever it fits the debug capacity;
+  * top-k stage: the number of ids kept is equal in every row, and for rows with an
+    active top-k (1 <= k < V, or greedy) the id set is bit-exact wherever it fits the
+    debug capacity;
   * logprob: |gpu - oracle| <= LOGPROB_TOL (absolute) against the primary result;
   * token: identical to the primary result, except *excused* rows: the GPU's
     (token, logprob) matches one of the results the definition gives when ln(min_p) moves
@@ -56,7 +57,9 @@ def compare(w, gpu, oracle_out, dbg_cap: int = 0, name: str = "") -> ParityRepor
         if gpu.get("num_topk") is not None and int(gpu["num_topk"][b]) != int(rows["n_topk"][b]):
             rep.failures.append((b, "top-k stage size", int(gpu["num_topk"][b]), int(rows["n_topk"][b])))
             continue
-        if dbg_cap and gpu.get("dbg_topk_ids") is not None and oracle_out.topk_ids is not None \
+        k_b = int(w.top_k[b]) if w.top_k is not None else 0
+        topk_active = bool(rows["greedy"][b]) or (1 <= k_b < w.V)
+        if dbg_cap and topk_active and gpu.get("dbg_topk_ids") is not None and oracle_out.topk_ids is not None \
                 and int(rows["n_topk"][b]) <= dbg_cap:
             g = np.sort(gpu["dbg_topk_ids"][b][gpu["dbg_topk_ids"][b] >= 0])
             o = np.sort(oracle_out.topk_ids[b][oracle_out.topk_ids[b] >= 0])
