@@ -60,6 +60,7 @@ enum {
 #define ALBIREO_ROW_GENERAL_PATH 1u  /* informational: row took the multi-pass general path */
 #define ALBIREO_ROW_BAD_PARAM 2u     /* T < 0 or NaN, r <= 0, ...: row treated per the clamps */
 #define ALBIREO_ROW_HISTORY_OVERFLOW 4u /* history did not fit the workspace: penalties skipped */
+#define ALBIREO_ROW_TIMEOUT 8u       /* a bounded on-chip wait expired: no result for this row   */
 
 /* flags of albireo_sample_ext_t.flags */
 #define ALBIREO_FLAG_FORCE_GENERAL 1u /* testing: send every row down the general path     */

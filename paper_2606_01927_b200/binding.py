@@ -19,7 +19,7 @@ from . import _build
 F32 = 0
 BF16 = 1
 OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED = 0, -1, -2, -3, -4
-ROW_GENERAL_PATH, ROW_BAD_PARAM, ROW_HISTORY_OVERFLOW = 1, 2, 4
+ROW_GENERAL_PATH, ROW_BAD_PARAM, ROW_HISTORY_OVERFLOW, ROW_TIMEOUT = 1, 2, 4, 8
 FLAG_FORCE_GENERAL = 1
 MAX_VOCAB = 524288
 MAX_NUM_TOP = 128

@@ -16,6 +16,7 @@
 // the order-preserving map of fp32 bit patterns.  Larger C comes first; all C distinct.
 // A kept set is always a prefix of that order, i.e. { t : C(t) >= threshold }.
 
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -24,6 +25,8 @@
 #include <new>
 
 #include "albireo_sample.h"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -36,8 +39,11 @@ constexpr int CNT_CAP = 4096;           // on-chip slots for distinct history id
 constexpr int CAND_CAP = 2048;          // candidate buffer entries (candidate path)
 constexpr int SORT_MAX = 512;           // most candidates the final stage sorts (== NT)
 constexpr int KA_MAX = 256;             // largest top-k the candidate path takes
-constexpr int TILE_VECS = 4;            // 16-byte vectors per thread per tile
-constexpr double FX50 = 1125899906842624.0;        // 2^50: fixed-point scale of the final stage
+constexpr int TILE_VECS = 2;            // 16-byte vectors per thread per tile
+constexpr int STAGE_BYTES = NT * TILE_VECS * 16;   // one ring stage = one tile (16 KiB)
+constexpr int MAX_STAGES = 8;
+constexpr int WAIT_CAP = 1 << 20;       // mbarrier polls before a wait gives up
+constexpr int COMMON_BYTES = 24576;     // histograms / candidate list, shared by the two paths
 constexpr uint32_t KEY_MIN_FINITE = 0x00800000u;   // key(-FLT_MAX); key(-inf) is one below
 constexpr uint32_t KEY_POS_INF = 0xFF800000u;      // key(+inf)
 constexpr float FX_SCALE = 1099511627776.0f;       // 2^40: fixed-point scale of masses
@@ -64,6 +70,7 @@ struct SampleArgs {
     int32_t dbg_cap;
     int32_t *dbg_topk_ids;
     uint32_t *out_row_status;
+    int32_t nstages;            // ring depth chosen by the host for this launch
     uint32_t *ws_counts;        // global scratch for history counts of rows with many distinct ids
     int64_t ws_counts_cap;      // entries
 };
@@ -111,11 +118,6 @@ __device__ __forceinline__ float neg_log_exp1_f32(uint32_t w) {
     }
     return -logf(E);
 }
-__device__ __forceinline__ double neg_log_exp1_f64(uint32_t w) {
-    double v = ((double)w + 0.5) * (1.0 / 4294967296.0);
-    return -log(-log1p(-v));
-}
-
 __device__ __forceinline__ uint32_t orderable_f32(float g) { return key_of(g); }
 
 // fixed-point mass of an element at distance d = z - zmax <= 0 (deterministic integer sums)
@@ -132,7 +134,8 @@ struct BlockScratch {
     uint32_t found_digit, found_cnt;
     u64 found_above;
     uint32_t list_cnt;
-    uint32_t cand_cnt, overflow, runmax;
+    uint32_t cand_cnt, overflow, runmax, timeout;
+    uint32_t r32a[NWARPS], r32b[NWARPS];
 };
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -591,90 +594,172 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
 }
 
 
+
+// ------------------------------------------------------------------ TMA bulk-copy ring
+//
+// The row is streamed through a ring of shared-memory stages filled by 1-D bulk async
+// copies (cp.async.bulk, completion on an mbarrier), several tiles ahead of the scan.
+// Every wait is bounded: on expiry the row reports ALBIREO_ROW_TIMEOUT and the CTA drains
+// its copies and leaves.
+
+struct Ring {
+    unsigned char *buf;     // nstages * STAGE_BYTES, 128-byte aligned
+    uint64_t *bar;          // one mbarrier per stage
+    int nstages;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+    for (int it = 0; it < WAIT_CAP; ++it) if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy; src and dst 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// issues the copy of tile t (called by one thread)
+__device__ __forceinline__ void ring_issue(const Ring &rg, const uint4 *vp, int nvec, int t) {
+    const int st = t % rg.nstages;
+    const int v0 = t * (NT * TILE_VECS);
+    int nv = nvec - v0; if (nv > NT * TILE_VECS) nv = NT * TILE_VECS;
+    mbar_expect_tx(&rg.bar[st], (uint32_t)nv * 16u);
+    bulk_g2s(rg.buf + (size_t)st * STAGE_BYTES, vp + v0, (uint32_t)nv * 16u, &rg.bar[st]);
+}
+// waits for the copies of tiles [t0, t1) so that the CTA may leave or reuse the ring
+__device__ void ring_drain(const Ring &rg, int t0, int t1) {
+    for (int t = t0; t < t1; ++t) mbar_wait(&rg.bar[t % rg.nstages], (uint32_t)(t / rg.nstages) & 1u);
+}
+
 // ------------------------------------------------------------------ candidate path
 //
 // One streaming pass over the row.  A conservative threshold tau (an order key) is kept
-// such that every element of the final kept set has key >= tau: the k-th largest key
-// among the candidates seen so far (top-k), and/or the min-p floor below the running
-// maximum.  Elements below tau are dropped by a cheap vector test; the rest are checked
-// exactly and appended to a small on-chip candidate list, which is then sorted and cut.
+// such that every element of the final kept set has key >= tau: (a lower bound of) the
+// k-th largest key seen so far (top-k), and/or the min-p floor below the running maximum.
+// Elements below tau are dropped by a cheap vector test; the rest are checked exactly and
+// appended to a small on-chip candidate list, which is finally sorted and cut.
 // Penalised tokens never enter through the stream (their raw value is not their score):
 // they are evaluated from the history bitmap after the stream.
 
 struct CandSmem {
-    u64 *cand;        // CAND_CAP composites
-    u64 *sorted;      // SORT_MAX composites, best first
-    uint32_t *hist;   // 256 bins
+    u64 *cand;        // CAND_CAP composites; after the sort: fixed-point masses of the sorted list
+    uint32_t *hist;   // SEL_BINS bins while selecting ...
+    u64 *sorted;      // ... SORT_MAX composites (best first) afterwards: same memory
 };
 
-__device__ __forceinline__ void cand_append(BlockScratch &s, u64 *cand, u64 C) {
-    uint32_t slot = atomicAdd(&s.cand_cnt, 1u);
-    if (slot < (uint32_t)CAND_CAP) cand[slot] = C; else s.overflow = 1u;
-    atomicMax(&s.runmax, (uint32_t)(C >> 32));
+constexpr int SEL_BINS = NT;            // one bin per thread
+
+__device__ __forceinline__ uint32_t warp_incl_scan_u32(uint32_t v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, o); if (lane >= o) v += t; }
+    return v;
 }
 
-// k-th largest key (1-based) among cand[0..n), n >= k: 8-bit radix select.  Uniform result.
-__device__ uint32_t cand_select_key(BlockScratch &s, const CandSmem &cs, int n, int k) {
-    uint32_t prefix = 0;
-    uint32_t rank = (uint32_t)k;
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        if (threadIdx.x < 256) cs.hist[threadIdx.x] = 0;
-        __syncthreads();
-        for (int i = threadIdx.x; i < n; i += NT) {
-            uint32_t key = (uint32_t)(cs.cand[i] >> 32);
-            if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&cs.hist[(key >> shift) & 255u], 1u);
-        }
-        __syncthreads();
-        if (threadIdx.x < 32) {
-            const int lane = threadIdx.x;
-            uint32_t local = 0;
+// block-wide max and min of 32-bit keys (ignore_zero: zeros do not take part in the min)
+__device__ void block_minmax_u32(BlockScratch &s, uint32_t v, uint32_t &mn, uint32_t &mx) {
+    uint32_t wmx = __reduce_max_sync(0xFFFFFFFFu, v);
+    uint32_t wmn = __reduce_min_sync(0xFFFFFFFFu, v ? v : 0xFFFFFFFFu);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) { s.r32a[threadIdx.x >> 5] = wmx; s.r32b[threadIdx.x >> 5] = wmn; }
+    __syncthreads();
+    uint32_t a = s.r32a[0], bmin = s.r32b[0];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) local += cs.hist[255 - (lane * 8 + q)];
-            uint32_t inc = local;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
-            uint32_t run = inc - local;
-            if (run < rank && rank <= run + local) {
-                for (int q = 0; q < 8; ++q) {
-                    uint32_t v = cs.hist[255 - (lane * 8 + q)];
-                    if (rank <= run + v) { s.found_digit = 255 - (lane * 8 + q); s.found_above = run; break; }
-                    run += v;
-                }
-            }
-        }
-        __syncthreads();
-        rank -= (uint32_t)s.found_above;
-        prefix = (prefix << 8) | s.found_digit;
+    for (int w = 1; w < NWARPS; ++w) { a = max(a, s.r32a[w]); bmin = min(bmin, s.r32b[w]); }
+    mx = a; mn = bmin;
+}
+
+// One histogram pass over cand[0..n) restricted to keys in [lo, hi]: finds the bin that
+// holds the k-th largest such key.  Returns false if fewer than k keys are in range.
+// On success [lo, hi] is narrowed to that bin and k to the rank inside it; `shift` tells
+// the bin width (0: the bin is a single key, i.e. lo is exactly the k-th largest key).
+__device__ bool cand_select_pass(BlockScratch &s, const CandSmem &cs, int n, uint32_t &k, uint32_t &lo, uint32_t &hi, int &shift) {
+    const uint32_t width = hi - lo;
+    shift = width < (uint32_t)SEL_BINS ? 0 : (32 - __clz(width)) - 9;
+    cs.hist[threadIdx.x] = 0;
+    if (threadIdx.x == 0) s.found_digit = 0xFFFFFFFFu;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += NT) {
+        uint32_t key = (uint32_t)(cs.cand[i] >> 32);
+        if (key >= lo && key <= hi) atomicAdd(&cs.hist[(key - lo) >> shift], 1u);
     }
-    return prefix;
+    __syncthreads();
+    // thread t owns bin SEL_BINS-1-t, so thread order is descending key order
+    const uint32_t mine = cs.hist[SEL_BINS - 1 - threadIdx.x];
+    const uint32_t inc = warp_incl_scan_u32(mine);
+    if ((threadIdx.x & 31) == 31) s.r32a[threadIdx.x >> 5] = inc;
+    __syncthreads();
+    uint32_t base = 0;
+    const int wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int w = 0; w < NWARPS; ++w) base += (w < wid) ? s.r32a[w] : 0u;
+    const uint32_t above = base + inc - mine;
+    if (above < k && k <= above + mine) { s.found_digit = SEL_BINS - 1 - threadIdx.x; s.found_cnt = above; }
+    __syncthreads();
+    const uint32_t digit = s.found_digit;
+    if (digit == 0xFFFFFFFFu) return false;
+    k -= s.found_cnt;
+    const uint32_t nlo = lo + (digit << shift);
+    uint32_t nhi = nlo + ((1u << shift) - 1u);
+    if (nhi > hi || nhi < nlo) nhi = hi;
+    lo = nlo; hi = nhi;
+    return true;
 }
 
-// keeps the candidates with key >= tkey; returns the new count (uniform)
+// Lower bound t of the k-th largest key in [lo, hi]: count(key >= t) >= k.  One pass.
+__device__ uint32_t cand_select_approx(BlockScratch &s, const CandSmem &cs, int n, int k, uint32_t lo, uint32_t hi) {
+    uint32_t kk = (uint32_t)k; int shift;
+    cand_select_pass(s, cs, n, kk, lo, hi, shift);     // on failure lo is unchanged: keep all
+    return lo;
+}
+// The k-th largest key in [lo, hi] exactly (as many passes as the key range needs).
+__device__ uint32_t cand_select_exact(BlockScratch &s, const CandSmem &cs, int n, int k, uint32_t lo, uint32_t hi) {
+    uint32_t kk = (uint32_t)k; int shift = 1;
+    for (int pass = 0; pass < 5 && shift != 0; ++pass)
+        if (!cand_select_pass(s, cs, n, kk, lo, hi, shift)) break;
+    return lo;
+}
+
+// keeps the candidates with key >= tkey (and drops empty slots); returns the new count
 __device__ int cand_compact(BlockScratch &s, const CandSmem &cs, int n, uint32_t tkey) {
     constexpr int PER = CAND_CAP / NT;
     u64 mine[PER];
+    uint32_t cnt = 0;
 #pragma unroll
     for (int q = 0; q < PER; ++q) {
         int i = threadIdx.x + q * NT;
         mine[q] = (i < n) ? cs.cand[i] : 0ull;
+        if ((uint32_t)(mine[q] >> 32) < tkey) mine[q] = 0ull;
+        cnt += mine[q] != 0ull;
     }
+    const uint32_t inc = warp_incl_scan_u32(cnt);
     __syncthreads();
     if (threadIdx.x == 0) s.cand_cnt = 0;
     __syncthreads();
+    uint32_t base = 0;
+    if ((threadIdx.x & 31) == 31 && inc) base = atomicAdd(&s.cand_cnt, inc);
+    base = __shfl_sync(0xFFFFFFFFu, base, 31) + inc - cnt;
 #pragma unroll
-    for (int q = 0; q < PER; ++q) {
-        if ((uint32_t)(mine[q] >> 32) >= tkey && mine[q] != 0ull) {
-            uint32_t slot = atomicAdd(&s.cand_cnt, 1u);
-            cs.cand[slot] = mine[q];
-        }
-    }
+    for (int q = 0; q < PER; ++q) if (mine[q] != 0ull) cs.cand[base++] = mine[q];
     __syncthreads();
     return (int)s.cand_cnt;
 }
 
-// Vector pre-test per dtype.  RawThr is the threshold in the domain the test runs in:
-// bf16: the smallest raw bf16 whose score has key >= tau (packed twice); fp32: unkey(tau).
+// Vector pre-test per dtype, in the domain the test runs in.
+// bf16: raw logits; the threshold is the smallest raw bf16 whose score has key >= tau
+// (packed twice).  fp32: scores; the threshold is unkey(tau).
 template <int DT> struct VecTest;
 template <> struct VecTest<ALBIREO_BF16> {
     static __device__ uint32_t raw_threshold(uint32_t tau_key, float invT) {
@@ -696,44 +781,167 @@ template <> struct VecTest<ALBIREO_BF16> {
         const uint32_t b = ok ? bits_of(k16) : 0xFF80u;     // not settled: let everything through
         return b | (b << 16);
     }
-    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
+    static __device__ __forceinline__ __nv_bfloat162 vmax(const uint4 &q) {
         __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x), *reinterpret_cast<const __nv_bfloat162 *>(&q.y));
         __nv_bfloat162 b2 = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&q.z), *reinterpret_cast<const __nv_bfloat162 *>(&q.w));
-        a = __hmax2(a, b2);
-        return __hge2_mask(a, *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
+        return __hmax2(a, b2);
+    }
+    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
+        return __hge2_mask(vmax(q), *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
+    }
+    // key of the score of the vector's largest element (an element of the row)
+    static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) {
+        __nv_bfloat162 m = vmax(q);
+        return key_of(__fmul_rn(fmaxf(__low2float(m), __high2float(m)), invT));
     }
     static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
 };
 template <> struct VecTest<ALBIREO_F32> {
     static __device__ uint32_t raw_threshold(uint32_t tau_key, float) { return __float_as_uint(unkey(tau_key)); }
-    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float invT) {
-        float m = fmaxf(fmaxf(__fmul_rn(__uint_as_float(q.x), invT), __fmul_rn(__uint_as_float(q.y), invT)),
-                        fmaxf(__fmul_rn(__uint_as_float(q.z), invT), __fmul_rn(__uint_as_float(q.w), invT)));
-        return m >= __uint_as_float(thr);
+    static __device__ __forceinline__ float vmaxz(const uint4 &q, float invT) {
+        return fmaxf(fmaxf(__fmul_rn(__uint_as_float(q.x), invT), __fmul_rn(__uint_as_float(q.y), invT)),
+                     fmaxf(__fmul_rn(__uint_as_float(q.z), invT), __fmul_rn(__uint_as_float(q.w), invT)));
     }
+    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float invT) {
+        return vmaxz(q, invT) >= __uint_as_float(thr);
+    }
+    static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) { return key_of(vmaxz(q, invT)); }
     static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
 };
 
-// exact check of one vector's unpenalised elements against tau; appends survivors
+// bit e set: element e of the vector is unpenalised and its score has key >= tau
 template <int DT>
-__device__ __noinline__ void slow_vector(BlockScratch &s, u64 *cand, const RowCtx &c, uint4 q, int i0,
-                                         uint32_t tau_key, u64 skip) {
+__device__ __forceinline__ uint32_t exact_pass_bits(const RowCtx &c, const uint4 &q, int i0, uint32_t tau_key) {
     typedef Elem<DT> E;
-    uint32_t m = 0;
+    uint32_t m = 0, bits = 0;
     if (c.has_hist) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+#pragma unroll
+    for (int e = 0; e < E::PER_VEC; ++e) {
+        uint32_t key = key_of(__fmul_rn(E::get(q, e), c.invT));
+        if (key >= tau_key && !((m >> e) & 1u)) bits |= 1u << e;
+    }
+    return bits;
+}
+
+// key of the largest unpenalised score in a vector (0 if none), for the warm-up bound
+template <int DT>
+__device__ __noinline__ uint32_t masked_vmax_key(const RowCtx &c, uint4 q, int i0) {
+    typedef Elem<DT> E;
+    const uint32_t m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+    uint32_t best = 0;
 #pragma unroll
     for (int e = 0; e < E::PER_VEC; ++e) {
         if (m & (1u << e)) continue;
         uint32_t key = key_of(__fmul_rn(E::get(q, e), c.invT));
-        u64 C = comp_of(key, i0 + e);
-        if (key >= tau_key && C != skip) cand_append(s, cand, C);
+        best = key > best ? key : best;
+    }
+    return best;
+}
+
+// Single appends outside the streaming loop (scalar head/tail, penalised tokens).
+__device__ __forceinline__ void cand_append_one(BlockScratch &s, u64 *cand, u64 C) {
+    cg::coalesced_group g = cg::coalesced_threads();
+    uint32_t base = 0;
+    if (g.thread_rank() == 0) base = atomicAdd(&s.cand_cnt, g.size());
+    base = g.shfl(base, 0);
+    const uint32_t slot = base + g.thread_rank();
+    if (slot < (uint32_t)CAND_CAP) cand[slot] = C; else s.overflow = 1u;
+}
+
+// Cuts and draw over the sorted candidate list, by one warp (no block barriers).
+// sorted[0..n) best first; efx: scratch for n fixed-point masses.
+__device__ void final_stage_warp(const u64 *sorted, u64 *efx, int n, int L6, bool has_minp, const RowParams &rp,
+                                 const SampleArgs &a, int b, RowOut &out) {
+    const int lane = threadIdx.x & 31;
+    const float zmax = unkey((uint32_t)(sorted[0] >> 32));
+    // min-p: a prefix; at least one survivor
+    int L7 = L6;
+    if (has_minp) {
+        const double ln_minp = log((double)rp.min_p);
+        int cnt = 0;
+        for (int j = lane; j < L6; j += 32) {
+            const double dj = (double)unkey((uint32_t)(sorted[j] >> 32)) - (double)zmax;
+            cnt += dj >= ln_minp;
+        }
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        L7 = cnt < 1 ? 1 : cnt;
+    }
+    // masses in fixed point (integer sums are exact, so the prefix sums are order-independent)
+    u64 tot = 0;
+    for (int j = lane; j < L7; j += 32) {
+        const float d = __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax);
+        const u64 e = mass_fx(d);
+        efx[j] = e;
+        tot += e;
+    }
+    tot = warp_sum_u64(tot);
+    __syncwarp();
+    int L8 = L7;
+    u64 S_fx = tot;
+    if (!rp.greedy && rp.top_p < 1.0f) {
+        double t = ceil((double)rp.top_p * (double)tot);
+        u64 target = t <= 1.0 ? 1ull : (u64)t;
+        if (target > tot) target = tot;
+        // smallest prefix whose mass reaches the target
+        u64 carry = 0;
+        int keepn = 0;
+        u64 kept_mass = 0;
+        for (int j0 = 0; j0 < L7; j0 += 32) {
+            const int j = j0 + lane;
+            const u64 e = j < L7 ? efx[j] : 0ull;
+            u64 inc = e;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t2; }
+            const u64 before = carry + inc - e;
+            const bool keep = j < L7 && before < target;
+            const uint32_t mk = __ballot_sync(0xFFFFFFFFu, keep);
+            keepn += __popc(mk);
+            if (mk) {
+                const int last = 31 - __clz(mk);
+                kept_mass = carry + __shfl_sync(0xFFFFFFFFu, inc, last);
+            }
+            carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
+            if (mk != 0xFFFFFFFFu) break;           // warp-uniform
+        }
+        L8 = keepn; S_fx = kept_mass;
+    }
+    const float lnS = logf((float)S_fx * (1.0f / FX_SCALE));
+    // race over the kept prefix
+    int tok = comp_idx(sorted[0]);
+    float lp_tok = 0.0f;
+    if (L8 > 1) {
+        u64 best = 0;
+        for (int j = lane; j < L8; j += 32) {
+            const int id = comp_idx(sorted[j]);
+            const float d = __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax);
+            const float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, id));
+            const u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)id);
+            best = G > best ? G : best;
+        }
+        best = warp_max_u64(best);
+        tok = comp_idx(best);
+        // logprob of the winner: find it in the list
+        float lp = 0.0f; bool mine = false;
+        for (int j = lane; j < L8; j += 32)
+            if (comp_idx(sorted[j]) == tok) { mine = true; lp = __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax) - lnS; }
+        const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
+        lp_tok = __shfl_sync(0xFFFFFFFFu, lp, __ffs(who) - 1);
+    }
+    out.token = tok; out.logprob = lp_tok; out.n_keep = L8;
+    if (a.num_top > 0) {
+        for (int j = lane; j < a.num_top && j < L8; j += 32) {
+            const int64_t q = (int64_t)b * a.num_top + j;
+            a.out_top_ids[q] = comp_idx(sorted[j]);
+            a.out_top_logprobs[q] = (L8 == 1) ? 0.0f : __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax) - lnS;
+        }
     }
 }
 
-// Returns false if the row must be handled by the general path instead.
+// Returns false if the row must be handled by the general path instead.  On success the
+// results are in `out` for warp 0 only (the other warps return early).
 template <int DT>
-__device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const RowCtx &c, const RowParams &rp,
-                               const SampleArgs &a, int b, RowOut &out) {
+__device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &rg, const RowCtx &c,
+                               const RowParams &rp, const SampleArgs &a, int b, RowOut &out) {
     typedef Elem<DT> E;
     typedef VecTest<DT> T;
     const int V = c.V;
@@ -745,10 +953,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const RowCtx
     // with the debug id list requested, keep the stream's threshold purely top-k so that the
     // top-k stage's set is known exactly
     const bool stream_minp = has_minp && !(has_topk && a.dbg_topk_ids != nullptr);
-    const double ln_minp = has_minp ? log((double)rp.min_p) : 0.0;
-
-    if (threadIdx.x == 0) { s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; }
-    __syncthreads();
+    const int lane = threadIdx.x & 31;
 
     const uintptr_t addr = (uintptr_t)c.row;
     int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
@@ -757,82 +962,138 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const RowCtx
     const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
     const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
 
-    uint32_t tau_key = KEY_MIN_FINITE;
-    uint32_t thr = T::raw_threshold(tau_key, c.invT);
-    uint32_t seen_max = 0;
-
-    auto floor_from_max = [&](uint32_t maxkey) -> uint32_t {
-        // a key no larger than the key of the smallest score that passes min-p under this maximum
-        return minp_key(unkey(maxkey), rp.min_p);
-    };
-
-    uint4 cur[TILE_VECS], nxt[TILE_VECS];
-#pragma unroll
-    for (int u = 0; u < TILE_VECS; ++u) {
-        int v = u * NT + threadIdx.x;
-        cur[u] = (v < nvec) ? __ldg(vp + v) : T::fill();
+    if (threadIdx.x == 0) {
+        s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
+        for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
+        for (int t = 0; t < npre; ++t) ring_issue(rg, vp, nvec, t);
     }
+    __syncthreads();
+
+    uint32_t tau_key = KEY_MIN_FINITE;
+    uint32_t thr = 0;
+    uint32_t seen_max = 0;
+    const uint32_t trig0 = has_topk ? (uint32_t)min(CAND_CAP / 2, 4 * k + 64) : (uint32_t)(CAND_CAP / 2);
+    uint32_t trig = trig0;
+
     for (int tile = 0; tile < ntiles; ++tile) {
         const int vbase = tile * NT * TILE_VECS;
-        if (tile + 1 < ntiles) {
+        const int st = tile % rg.nstages;
+        bool flag = false;
+        if (!mbar_wait(&rg.bar[st], (uint32_t)(tile / rg.nstages) & 1u)) { s.timeout = 1u; flag = true; }
+        const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES);
+        uint4 cur[TILE_VECS];
 #pragma unroll
-            for (int u = 0; u < TILE_VECS; ++u) {
-                int v = vbase + NT * TILE_VECS + u * NT + threadIdx.x;
-                nxt[u] = (v < nvec) ? __ldg(vp + v) : T::fill();
-            }
+        for (int u = 0; u < TILE_VECS; ++u) {
+            const int vl = u * NT + threadIdx.x;
+            cur[u] = (vbase + vl < nvec && !flag) ? stage[vl] : T::fill();
         }
-        u64 own = 0;
         if (tile == 0) {
-            // warm-up: every thread contributes its best unpenalised element; the k-th largest
-            // of these is a valid lower bound of the row's k-th largest score
+            // warm-up: the k-th largest of the per-thread maxima (each an unpenalised element of
+            // the row, all distinct) is a lower bound of the row's k-th largest score
+            uint32_t mk = 0;
 #pragma unroll
             for (int u = 0; u < TILE_VECS; ++u) {
-                const int i0 = head + (vbase + u * NT + threadIdx.x) * E::PER_VEC;
-                uint32_t m = 0;
-                if (c.has_hist && i0 < V) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
-#pragma unroll
-                for (int e = 0; e < E::PER_VEC; ++e) {
-                    uint32_t key = key_of(__fmul_rn(E::get(cur[u], e), c.invT));
-                    u64 C = comp_of(key, i0 + e);
-                    if (!(m & (1u << e)) && key >= KEY_MIN_FINITE && C > own) own = C;
+                const int v = u * NT + threadIdx.x;
+                if (v < nvec) {
+                    const int i0 = head + v * E::PER_VEC;
+                    uint32_t kk;
+                    if (c.has_hist && (__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u)))
+                        kk = masked_vmax_key<DT>(c, cur[u], i0);
+                    else
+                        kk = T::vmax_key(cur[u], c.invT);
+                    mk = kk > mk ? kk : mk;
                 }
             }
-            if (own) cand_append(s, cs.cand, own);
-            __syncthreads();
-            int n = (int)s.cand_cnt;
-            uint32_t rmax = s.runmax;
-            __syncthreads();
-            if (has_topk && n >= k) tau_key = cand_select_key(s, cs, n, k);
-            if (stream_minp && rmax) { uint32_t f = floor_from_max(rmax); tau_key = f > tau_key ? f : tau_key; }
-            seen_max = rmax;
+            if (mk < KEY_MIN_FINITE || mk >= KEY_POS_INF) mk = 0;
+            cs.cand[threadIdx.x] = (u64)mk << 32;
+            const int valid = __syncthreads_count(mk != 0);
+            uint32_t kmin, kmax;
+            block_minmax_u32(s, mk, kmin, kmax);
+            if (stream_minp && threadIdx.x == 0) s.runmax = kmax;
+            if (has_topk && valid >= k) tau_key = cand_select_approx(s, cs, NT, k, kmin, kmax);
+            if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
+            seen_max = kmax;
             thr = T::raw_threshold(tau_key, c.invT);
+            __syncthreads();
         }
+        // scan: cheap vector test, then the exact element test for vectors that may pass
+        uint32_t bits[TILE_VECS];
+        uint32_t cnt = 0;
 #pragma unroll
         for (int u = 0; u < TILE_VECS; ++u) {
             const int v = vbase + u * NT + threadIdx.x;
-            if (v < nvec && T::may_pass(cur[u], thr, c.invT))
-                slow_vector<DT>(s, cs.cand, c, cur[u], head + v * E::PER_VEC, tau_key, own);
+            bits[u] = 0;
+            if (v < nvec && T::may_pass(cur[u], thr, c.invT)) bits[u] = exact_pass_bits<DT>(c, cur[u], head + v * E::PER_VEC, tau_key);
+            cnt += __popc(bits[u]);
         }
-        __syncthreads();                       // every append of this tile is done
-        int n = (int)s.cand_cnt;
-        const uint32_t ovf = s.overflow, rmax = s.runmax;
-        __syncthreads();                       // nobody appends again before all have read
-        if (ovf) return false;
-        bool changed = false;
-        if (has_topk && n >= k && (n >= 2 * k + 32 || n > CAND_CAP / 2 || tile == 0)) {
-            uint32_t t = cand_select_key(s, cs, n, k);
-            if (t > tau_key) { tau_key = t; changed = true; }
-            n = cand_compact(s, cs, n, tau_key);
-        }
-        if (stream_minp && rmax != seen_max) {
-            seen_max = rmax;
-            uint32_t f = floor_from_max(rmax);
-            if (f > tau_key) { tau_key = f; changed = true; }
-        }
-        if (!has_topk && n > CAND_CAP / 2) n = cand_compact(s, cs, n, tau_key);
-        if (changed) thr = T::raw_threshold(tau_key, c.invT);
+        if (__any_sync(0xFFFFFFFFu, cnt != 0)) {
+            // one reservation per warp, then every lane writes its survivors
+            const uint32_t inc = warp_incl_scan_u32(cnt);
+            const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            uint32_t base = 0;
+            if (lane == 31) base = atomicAdd(&s.cand_cnt, total);
+            base = __shfl_sync(0xFFFFFFFFu, base, 31);
+            flag = flag || base + total + 1u >= trig;
+            if (base + total > (uint32_t)CAND_CAP) { if (lane == 31) s.overflow = 1u; flag = true; }
+            else {
+                uint32_t slot = base + inc - cnt;
+                uint32_t lmax = 0;
 #pragma unroll
-        for (int u = 0; u < TILE_VECS; ++u) cur[u] = nxt[u];
+                for (int u = 0; u < TILE_VECS; ++u) {
+                    const int i0 = head + (vbase + u * NT + threadIdx.x) * E::PER_VEC;
+#pragma unroll
+                    for (int e = 0; e < E::PER_VEC; ++e) {
+                        if ((bits[u] >> e) & 1u) {
+                            const uint32_t key = key_of(__fmul_rn(E::get(cur[u], e), c.invT));
+                            cs.cand[slot++] = comp_of(key, i0 + e);
+                            lmax = key > lmax ? key : lmax;
+                        }
+                    }
+                }
+                if (stream_minp) {
+                    lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
+                    if (lane == 0 && lmax > seen_max) { uint32_t old = atomicMax(&s.runmax, lmax); flag = flag || lmax > old; }
+                }
+            }
+        }
+        const bool need = __syncthreads_or(flag);      // also: every thread is done reading this stage
+        if (threadIdx.x == 0 && tile + rg.nstages < ntiles && !s.timeout) ring_issue(rg, vp, nvec, tile + rg.nstages);
+        if (need) {
+            // every thread is here, so nobody appends until the barriers below are passed
+            int n = (int)s.cand_cnt;
+            const uint32_t ovf = s.overflow, rmax = s.runmax, tmo = s.timeout;
+            __syncthreads();
+            if (ovf || tmo) {
+                const int issued = min(ntiles, tile + 1 + rg.nstages);
+                ring_drain(rg, tmo ? tile : tile + 1, tmo ? min(ntiles, tile + rg.nstages) : issued);   // after a timeout nothing new was issued
+                if (tmo) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; return true; }
+                __syncthreads();
+                return false;
+            }
+            bool changed = false;
+            if (stream_minp && rmax > seen_max) {
+                seen_max = rmax;
+                uint32_t f = minp_key(unkey(rmax), rp.min_p);
+                if (f > tau_key) { tau_key = f; changed = true; }
+            }
+            if ((uint32_t)n + 1u >= trig) {
+                if (has_topk && n >= k) {
+                    uint32_t lmx = 0, mn, hi;
+                    for (int i = threadIdx.x; i < n; i += NT) { uint32_t kk = (uint32_t)(cs.cand[i] >> 32); lmx = kk > lmx ? kk : lmx; }
+                    block_minmax_u32(s, lmx, mn, hi);
+                    uint32_t t = cand_select_approx(s, cs, n, k, tau_key, hi);
+                    if (t > tau_key) { tau_key = t; changed = true; }
+                }
+                n = cand_compact(s, cs, n, tau_key);
+                // if the list could not be shrunk (ties), look again only after it has grown
+                trig = (uint32_t)n + (uint32_t)(has_topk ? 2 * k + 32 : CAND_CAP / 4);
+                if (trig < trig0) trig = trig0;
+            }
+            if (changed) thr = T::raw_threshold(tau_key, c.invT);
+        }
     }
     // scalar head and tail of a row that is not 16-byte aligned / not a whole number of vectors
     {
@@ -842,69 +1103,64 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const RowCtx
             int i = q < head ? q : tail0 + (q - head);
             if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
             uint32_t key = key_of(__fmul_rn(E::load(c.row, i), c.invT));
-            if (key >= tau_key) cand_append(s, cs.cand, comp_of(key, i));
+            if (key >= tau_key) cand_append_one(s, cs.cand, comp_of(key, i));
         }
     }
     // penalised tokens, straight from the history bitmap
     if (c.has_hist) {
         const int nwords = (V + 31) >> 5;
         for (int w = threadIdx.x; w < nwords; w += NT) {
-            uint32_t bits = c.bitmap[w];
-            if (!bits) continue;
+            uint32_t wbits = c.bitmap[w];
+            if (!wbits) continue;
             uint32_t r = c.coarse[w >> 3];
             for (int ww = (w >> 3) << 3; ww < w; ++ww) r += __popc(c.bitmap[ww]);
-            while (bits) {
-                int bit = __ffs(bits) - 1;
-                bits &= bits - 1;
+            while (wbits) {
+                int bit = __ffs(wbits) - 1;
+                wbits &= wbits - 1;
                 int i = (w << 5) + bit;
                 float x = E::load(c.row, i);
-                uint32_t cnt = c.counts[r++];
+                uint32_t cntv = c.counts[r++];
                 float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
-                av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cnt)));
+                av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cntv)));
                 av = __fsub_rn(av, c.p);
                 uint32_t key = key_of(__fmul_rn(av, c.invT));
-                if (key >= tau_key) cand_append(s, cs.cand, comp_of(key, i));
+                if (key >= tau_key) cand_append_one(s, cs.cand, comp_of(key, i));
             }
         }
     }
     __syncthreads();
     int n = (int)s.cand_cnt;
     const uint32_t ovf = s.overflow;
-    const uint32_t kmax = s.runmax;
     __syncthreads();
     if (ovf || n < 1) return false;
 
-    // exact top-k threshold, then the exact min-p floor for rows without a top-k
     bool topk_exact_known = true;      // is min(k, #finite) known without counting?
     if (has_topk) {
-        if (n > k) {
-            uint32_t t = cand_select_key(s, cs, n, k);
+        if (n > SORT_MAX || n > 2 * k + 96) {
+            uint32_t lmx = 0, mn, hi;
+            for (int i = threadIdx.x; i < n; i += NT) { uint32_t kk = (uint32_t)(cs.cand[i] >> 32); lmx = kk > lmx ? kk : lmx; }
+            block_minmax_u32(s, lmx, mn, hi);
+            uint32_t t = cand_select_exact(s, cs, n, k, tau_key, hi);
             n = cand_compact(s, cs, n, t);
-        } else if (n < k && stream_minp) {
-            topk_exact_known = false;
         }
+        if (n < k && stream_minp) topk_exact_known = false;
     } else {
-        n = cand_compact(s, cs, n, floor_from_max(kmax));
+        uint32_t lmx = 0, mn, hi;
+        for (int i = threadIdx.x; i < n; i += NT) { uint32_t kk = (uint32_t)(cs.cand[i] >> 32); lmx = kk > lmx ? kk : lmx; }
+        block_minmax_u32(s, lmx, mn, hi);
+        n = cand_compact(s, cs, n, minp_key(unkey(hi), rp.min_p));
         topk_exact_known = false;
     }
     if (n > SORT_MAX || n < 1) return false;
 
-    // sort by rank counting (all composites distinct)
+    // sort by rank counting (all composites distinct); `sorted` reuses the histogram memory
     if (threadIdx.x < n) {
         const u64 C = cs.cand[threadIdx.x];
         int rank = 0;
         for (int j = 0; j < n; ++j) rank += cs.cand[j] > C;
         cs.sorted[rank] = C;
     }
-    __syncthreads();
-
-    const int j = threadIdx.x;
-    const u64 Cj = j < n ? cs.sorted[j] : 0ull;
-    const float zmax = unkey((uint32_t)(cs.sorted[0] >> 32));
-    const float zj = unkey((uint32_t)(Cj >> 32));
-    const double dj = (double)zj - (double)zmax;
     const int L6 = has_topk ? (n < k ? n : k) : n;
-
     int n_topk = L6;
     if (!topk_exact_known && a.out_num_topk) {
         // diagnostic only: count the finite scores of the row
@@ -913,64 +1169,21 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const RowCtx
         u64 nfin = block_sum_u64(s, local);
         n_topk = has_topk ? (int)(nfin < (u64)k ? nfin : (u64)k) : (int)nfin;
     }
+    __syncthreads();
     out.n_topk = n_topk;
-    if (a.dbg_topk_ids && has_topk && L6 <= a.dbg_cap && j < L6) a.dbg_topk_ids[(int64_t)b * a.dbg_cap + j] = comp_idx(Cj);
-
-    // min-p (a prefix of the order), at least one survivor
-    bool in7 = j < L6 && (!has_minp || dj >= ln_minp);
-    int L7 = (int)block_sum_u64(s, in7 ? 1u : 0u);
-    if (L7 < 1) L7 = 1;
-    // top-p over the survivors' mass, fixed-point so that the sums do not depend on the order
-    u64 ej = (j < L7) ? __double2ull_rn(exp(dj) * FX50) : 0ull;
-    u64 total;
-    u64 before = block_exscan_u64(s, ej, total);
-    bool keep = j < L7;
-    if (!rp.greedy && rp.top_p < 1.0f) {
-        double t = ceil((double)rp.top_p * (double)total);
-        u64 target = t <= 1.0 ? 1ull : (u64)t;
-        if (target > total) target = total;
-        keep = keep && before < target;
-    }
-    const int L8 = (int)block_sum_u64(s, keep ? 1u : 0u);
-    const u64 S_fx = block_sum_u64(s, keep ? ej : 0ull);
-    const double lnS = log((double)S_fx) - 50.0 * 0.6931471805599453;
-    out.n_keep = L8;
-
-    // race
-    const int id = comp_idx(Cj);
-    u64 G = 0;
-    if (keep) {
-        double g = dj + neg_log_exp1_f64(race_word(rp.seed, rp.R, a.step, id));
-        long long gb = __double_as_longlong(g);
-        G = (gb < 0) ? ~(u64)gb : ((u64)gb | 0x8000000000000000ull);
-    }
-    const u64 Gmax = block_max_u64(s, G);
-    const u64 win = block_max_u64(s, (keep && G == Gmax) ? (u64)(uint32_t)(~(uint32_t)id) : 0ull);
-    const int tok = (L8 == 1) ? comp_idx(cs.sorted[0]) : (int)(~(uint32_t)win);
-    if (keep && id == tok) {
-        s.bcast[0] = (u64)__float_as_uint((L8 == 1) ? 0.0f : (float)(dj - lnS));
-    }
-    __syncthreads();
-    out.token = tok;
-    out.logprob = __uint_as_float((uint32_t)s.bcast[0]);
-    if (a.num_top > 0 && j < a.num_top) {
-        const int64_t q = (int64_t)b * a.num_top + j;
-        if (j < L8) {
-            a.out_top_ids[q] = id;
-            a.out_top_logprobs[q] = (L8 == 1) ? 0.0f : (float)(dj - lnS);
-        }
-    }
-    __syncthreads();
+    if (a.dbg_topk_ids && has_topk && L6 <= a.dbg_cap && threadIdx.x < L6)
+        a.dbg_topk_ids[(int64_t)b * a.dbg_cap + threadIdx.x] = comp_idx(cs.sorted[threadIdx.x]);
+    if (threadIdx.x < 32) final_stage_warp(cs.sorted, cs.cand, n, L6, has_minp, rp, a, b, out);
     return true;
 }
 
 // ------------------------------------------------------------------ the kernel
 
 // dynamic shared memory layout (bytes): [24 KiB shared by the two paths: histograms (cnt 8 KiB, mass
-// 16 KiB) or candidates (16 KiB) + sorted list (4 KiB) + 256 bins (1 KiB)][bitmap][coarse][counts]
+// 16 KiB) or candidates (16 KiB) + 2048 bins / sorted list (8 KiB)][bitmap][coarse][counts]
 template <int DT>
 __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs a) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     __shared__ BlockScratch s;
     const int b = blockIdx.x;
     const int V = a.V;
@@ -978,9 +1191,13 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     HistBins h;
     h.cnt = (uint32_t *)smem;
     h.mass = (u64 *)(smem + HIST_BINS * 4);
+    Ring rg;
+    rg.nstages = a.nstages;
+    rg.buf = smem + COMMON_BYTES;
+    rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
     HistSmem hs;
     const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
-    hs.bitmap = (uint32_t *)(smem + HIST_BINS * 12);
+    hs.bitmap = (uint32_t *)((unsigned char *)rg.bar + MAX_STAGES * 8);
     hs.coarse = hs.bitmap + (nwords + 1);
     hs.counts = hs.coarse + (ncoarse + 1);
 
@@ -1026,10 +1243,10 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
 
     CandSmem cs;
     cs.cand = (u64 *)smem;                                  // 16 KiB
-    cs.sorted = (u64 *)(smem + CAND_CAP * 8);               // 4 KiB
-    cs.hist = (uint32_t *)(smem + CAND_CAP * 8 + SORT_MAX * 8);   // 1 KiB
+    cs.hist = (uint32_t *)(smem + CAND_CAP * 8);            // 8 KiB while selecting ...
+    cs.sorted = (u64 *)(smem + CAND_CAP * 8);               // ... then the 4 KiB sorted list
     bool done = false;
-    if (!(a.flags & ALBIREO_FLAG_FORCE_GENERAL)) done = candidate_path<DT>(s, cs, c, rp, a, b, out);
+    if (!(a.flags & ALBIREO_FLAG_FORCE_GENERAL)) done = candidate_path<DT>(s, cs, rg, c, rp, a, b, out);
     if (!done) {
         __syncthreads();
         general_path<DT>(s, h, c, rp, a, b, out);
@@ -1044,13 +1261,23 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     }
 }
 
-size_t smem_bytes_for(int V, bool with_history) {
-    size_t bytes = (size_t)HIST_BINS * 12;
-    if (with_history) {
-        size_t nwords = ((size_t)V + 31) / 32, ncoarse = (nwords + 7) / 8;
-        bytes += (nwords + 1 + ncoarse + 1 + CNT_CAP) * 4;
-    }
-    return (bytes + 15) & ~(size_t)15;
+size_t history_smem_bytes(int V) {
+    size_t nwords = ((size_t)V + 31) / 32, ncoarse = (nwords + 7) / 8;
+    return (nwords + 1 + ncoarse + 1 + CNT_CAP) * 4;
+}
+// ring depth: as deep as lets two CTAs share an SM (228 KiB per SM, 1 KiB reserved per CTA)
+int ring_stages_for(int V, bool with_history) {
+    const long budget = (233472 / 2) - 1024 - 1024;      // per CTA: dynamic bytes available
+    long fixed = COMMON_BYTES + MAX_STAGES * 8 + (with_history ? (long)history_smem_bytes(V) : 0);
+    long n = (budget - fixed) / STAGE_BYTES;
+    if (n < 2) n = 2;
+    if (n > 6) n = 6;
+    return (int)n;
+}
+size_t smem_bytes_for(int V, bool with_history, int nstages) {
+    size_t bytes = (size_t)COMMON_BYTES + (size_t)nstages * STAGE_BYTES + MAX_STAGES * 8;
+    if (with_history) bytes += history_smem_bytes(V);
+    return (bytes + 127) & ~(size_t)127;
 }
 
 constexpr size_t WS_HEADER = 256;
@@ -1106,11 +1333,22 @@ extern "C" int albireo_sample_init(albireo_sampler_t **out, int32_t device, int3
     int prev = -1;
     if (cudaGetDevice(&prev) != cudaSuccess) return ALBIREO_ECUDA;
     if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return ALBIREO_ECUDA; }
-    const size_t smem = smem_bytes_for(max_vocab, true);
-    cudaError_t e1 = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    cudaError_t e2 = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // opt in to the largest dynamic shared memory a CTA may have on this device
+    int optin = 0;
+    cudaError_t e0 = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    cudaFuncAttributes fa32, fa16;
+    cudaError_t e1 = cudaFuncGetAttributes(&fa32, albireo_sample_kernel<ALBIREO_F32>);
+    cudaError_t e2 = cudaFuncGetAttributes(&fa16, albireo_sample_kernel<ALBIREO_BF16>);
+    size_t smem = 0;
+    if (e0 == cudaSuccess && e1 == cudaSuccess && e2 == cudaSuccess) {
+        const size_t stat = fa32.sharedSizeBytes > fa16.sharedSizeBytes ? fa32.sharedSizeBytes : fa16.sharedSizeBytes;
+        smem = (size_t)optin > stat ? (size_t)optin - stat : 0;
+        e1 = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e2 = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    }
     if (prev >= 0 && prev != device) cudaSetDevice(prev);
-    if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); return ALBIREO_ECUDA; }
+    if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); return ALBIREO_ECUDA; }
+    if (smem_bytes_for(max_vocab, true, 2) > smem) return ALBIREO_EUNSUPPORTED;
 
     albireo_sampler *h = new (std::nothrow) albireo_sampler();
     if (!h) return ALBIREO_ENOMEM;
@@ -1169,7 +1407,10 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
     int cur = -1;
     if (cudaGetDevice(&cur) != cudaSuccess || cur != h->device) { cudaGetLastError(); set_err(h, "the handle's device is not current%s", ""); return ALBIREO_EINVAL; }
 
-    const size_t smem = smem_bytes_for(V, history_ids != nullptr);
+    a.nstages = ring_stages_for(V, history_ids != nullptr);
+    size_t smem = smem_bytes_for(V, history_ids != nullptr, a.nstages);
+    while (smem > h->max_smem && a.nstages > 2) smem = smem_bytes_for(V, history_ids != nullptr, --a.nstages);
+    if (smem > h->max_smem) { set_err(h, "vocabulary too large for the on-chip tables%s", ""); return ALBIREO_EUNSUPPORTED; }
     cudaStream_t st = (cudaStream_t)stream;
     if (dtype == ALBIREO_F32) albireo_sample_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(a);
     else albireo_sample_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(a);
