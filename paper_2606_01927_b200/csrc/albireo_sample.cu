@@ -35,15 +35,15 @@ typedef unsigned long long u64;
 constexpr int NT = 512;                 // threads per CTA
 constexpr int NWARPS = NT / 32;
 constexpr int HIST_BINS = 2048;         // 11-bit digits
-constexpr int CNT_CAP = 4096;           // on-chip slots for distinct history ids per row
-constexpr int CAND_CAP = 2048;          // candidate buffer entries (candidate path)
+constexpr int CNT_CAP = 2048;           // on-chip slots for distinct history ids per row
+constexpr int CAND_CAP = 1024;          // candidate buffer entries (candidate path)
 constexpr int SORT_MAX = 512;           // most candidates the final stage sorts (== NT)
 constexpr int KA_MAX = 256;             // largest top-k the candidate path takes
-constexpr int TILE_VECS = 2;            // 16-byte vectors per thread per tile
-constexpr int STAGE_BYTES = NT * TILE_VECS * 16;   // one ring stage = one tile (16 KiB)
+constexpr int TILE_VECS = 4;            // 16-byte vectors per thread per tile
+constexpr int STAGE_BYTES = NT * TILE_VECS * 16;   // one ring stage = one tile (32 KiB)
 constexpr int MAX_STAGES = 8;
 constexpr int WAIT_CAP = 1 << 20;       // mbarrier polls before a wait gives up
-constexpr int COMMON_BYTES = 24576;     // histograms / candidate list, shared by the two paths
+constexpr int COMMON_BYTES = 12288;     // candidate list (8 KiB) + select bins / sorted list (4 KiB)
 constexpr uint32_t KEY_MIN_FINITE = 0x00800000u;   // key(-FLT_MAX); key(-inf) is one below
 constexpr uint32_t KEY_POS_INF = 0xFF800000u;      // key(+inf)
 constexpr float FX_SCALE = 1099511627776.0f;       // 2^40: fixed-point scale of masses
@@ -219,6 +219,8 @@ template <int DT> struct Elem;
 template <> struct Elem<ALBIREO_F32> {
     static constexpr int SIZE = 4, PER_VEC = 4;
     static __device__ __forceinline__ float load(const void *row, int i) { return __ldg((const float *)row + i); }
+    // plain load through a generic pointer (shared memory allowed)
+    static __device__ __forceinline__ float load_plain(const void *p, int i) { return ((const float *)p)[i]; }
     static __device__ __forceinline__ float get(const uint4 &q, int e) {
         return __uint_as_float(e == 0 ? q.x : e == 1 ? q.y : e == 2 ? q.z : q.w);
     }
@@ -227,6 +229,9 @@ template <> struct Elem<ALBIREO_BF16> {
     static constexpr int SIZE = 2, PER_VEC = 8;
     static __device__ __forceinline__ float load(const void *row, int i) {
         return __uint_as_float(((uint32_t)__ldg((const unsigned short *)row + i)) << 16);
+    }
+    static __device__ __forceinline__ float load_plain(const void *p, int i) {
+        return __uint_as_float(((uint32_t)((const unsigned short *)p)[i]) << 16);
     }
     static __device__ __forceinline__ float get(const uint4 &q, int e) {
         uint32_t w = (e >> 1) == 0 ? q.x : (e >> 1) == 1 ? q.y : (e >> 1) == 2 ? q.z : q.w;
@@ -631,8 +636,7 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 // issues the copy of tile t (called by one thread)
-__device__ __forceinline__ void ring_issue(const Ring &rg, const uint4 *vp, int nvec, int t) {
-    const int st = t % rg.nstages;
+__device__ __forceinline__ void ring_issue(const Ring &rg, const uint4 *vp, int nvec, int t, int st) {
     const int v0 = t * (NT * TILE_VECS);
     int nv = nvec - v0; if (nv > NT * TILE_VECS) nv = NT * TILE_VECS;
     mbar_expect_tx(&rg.bar[st], (uint32_t)nv * 16u);
@@ -789,6 +793,22 @@ template <> struct VecTest<ALBIREO_BF16> {
     static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
         return __hge2_mask(vmax(q), *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
     }
+    static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float) {
+        __nv_bfloat162 m = vmax(q[0]);
+#pragma unroll
+        for (int u = 1; u < TILE_VECS; ++u) m = __hmax2(m, vmax(q[u]));
+        return __hge2_mask(m, *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
+    }
+    // bit e set: raw element e >= the raw threshold (a superset of "score key >= tau")
+    static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float) {
+        const __nv_bfloat162 t2 = *reinterpret_cast<const __nv_bfloat162 *>(&thr);
+        const uint32_t r0 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.x), t2);
+        const uint32_t r1 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.y), t2);
+        const uint32_t r2 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.z), t2);
+        const uint32_t r3 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.w), t2);
+        return ((r0 & 1u) | ((r0 >> 15) & 2u)) | (((r1 & 1u) | ((r1 >> 15) & 2u)) << 2) |
+               (((r2 & 1u) | ((r2 >> 15) & 2u)) << 4) | (((r3 & 1u) | ((r3 >> 15) & 2u)) << 6);
+    }
     // key of the score of the vector's largest element (an element of the row)
     static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) {
         __nv_bfloat162 m = vmax(q);
@@ -804,6 +824,17 @@ template <> struct VecTest<ALBIREO_F32> {
     }
     static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float invT) {
         return vmaxz(q, invT) >= __uint_as_float(thr);
+    }
+    static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float invT) {
+        float m = vmaxz(q[0], invT);
+#pragma unroll
+        for (int u = 1; u < TILE_VECS; ++u) m = fmaxf(m, vmaxz(q[u], invT));
+        return m >= __uint_as_float(thr);
+    }
+    static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float invT) {
+        const float t = __uint_as_float(thr);
+        return (uint32_t)(__fmul_rn(__uint_as_float(q.x), invT) >= t) | ((uint32_t)(__fmul_rn(__uint_as_float(q.y), invT) >= t) << 1) |
+               ((uint32_t)(__fmul_rn(__uint_as_float(q.z), invT) >= t) << 2) | ((uint32_t)(__fmul_rn(__uint_as_float(q.w), invT) >= t) << 3);
     }
     static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) { return key_of(vmaxz(q, invT)); }
     static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
@@ -968,7 +999,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
-        for (int t = 0; t < npre; ++t) ring_issue(rg, vp, nvec, t);
+        for (int t = 0; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
     }
     __syncthreads();
 
@@ -978,17 +1009,21 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     const uint32_t trig0 = has_topk ? (uint32_t)min(CAND_CAP / 2, 4 * k + 64) : (uint32_t)(CAND_CAP / 2);
     uint32_t trig = trig0;
 
+    int st = 0;                      // ring stage of the current tile
+    uint32_t parity = 0;             // its mbarrier phase
     for (int tile = 0; tile < ntiles; ++tile) {
         const int vbase = tile * NT * TILE_VECS;
-        const int st = tile % rg.nstages;
         bool flag = false;
-        if (!mbar_wait(&rg.bar[st], (uint32_t)(tile / rg.nstages) & 1u)) { s.timeout = 1u; flag = true; }
-        const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES);
+        if (!mbar_wait(&rg.bar[st], parity)) { s.timeout = 1u; flag = true; }
+        const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + threadIdx.x;
         uint4 cur[TILE_VECS];
+        if (vbase + NT * TILE_VECS <= nvec && !flag) {
 #pragma unroll
-        for (int u = 0; u < TILE_VECS; ++u) {
-            const int vl = u * NT + threadIdx.x;
-            cur[u] = (vbase + vl < nvec && !flag) ? stage[vl] : T::fill();
+            for (int u = 0; u < TILE_VECS; ++u) cur[u] = stage[u * NT];
+        } else {
+#pragma unroll
+            for (int u = 0; u < TILE_VECS; ++u)
+                cur[u] = (vbase + u * NT + (int)threadIdx.x < nvec && !flag) ? stage[u * NT] : T::fill();
         }
         if (tile == 0) {
             // warm-up: the k-th largest of the per-thread maxima (each an unpenalised element of
@@ -1019,48 +1054,52 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             thr = T::raw_threshold(tau_key, c.invT);
             __syncthreads();
         }
-        // scan: cheap vector test, then the exact element test for vectors that may pass
-        uint32_t bits[TILE_VECS];
-        uint32_t cnt = 0;
+        // scan: one cheap test for the whole tile share of this thread; the exact element test
+        // only in warps where some vector may pass
+        if (__any_sync(0xFFFFFFFFu, T::any_may_pass(cur, thr, c.invT))) {
+            // per-element test in the test domain (a superset of key >= tau), minus penalised tokens
+            uint32_t all = 0;
 #pragma unroll
-        for (int u = 0; u < TILE_VECS; ++u) {
-            const int v = vbase + u * NT + threadIdx.x;
-            bits[u] = 0;
-            if (v < nvec && T::may_pass(cur[u], thr, c.invT)) bits[u] = exact_pass_bits<DT>(c, cur[u], head + v * E::PER_VEC, tau_key);
-            cnt += __popc(bits[u]);
-        }
-        if (__any_sync(0xFFFFFFFFu, cnt != 0)) {
-            // one reservation per warp, then every lane writes its survivors
-            const uint32_t inc = warp_incl_scan_u32(cnt);
-            const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            uint32_t base = 0;
-            if (lane == 31) base = atomicAdd(&s.cand_cnt, total);
-            base = __shfl_sync(0xFFFFFFFFu, base, 31);
-            flag = flag || base + total + 1u >= trig;
-            if (base + total > (uint32_t)CAND_CAP) { if (lane == 31) s.overflow = 1u; flag = true; }
-            else {
-                uint32_t slot = base + inc - cnt;
-                uint32_t lmax = 0;
-#pragma unroll
-                for (int u = 0; u < TILE_VECS; ++u) {
+            for (int u = 0; u < TILE_VECS; ++u) {
+                uint32_t bts = T::elem_bits(cur[u], thr, c.invT);
+                if (c.has_hist && bts) {
                     const int i0 = head + (vbase + u * NT + threadIdx.x) * E::PER_VEC;
-#pragma unroll
-                    for (int e = 0; e < E::PER_VEC; ++e) {
-                        if ((bits[u] >> e) & 1u) {
-                            const uint32_t key = key_of(__fmul_rn(E::get(cur[u], e), c.invT));
-                            cs.cand[slot++] = comp_of(key, i0 + e);
-                            lmax = key > lmax ? key : lmax;
-                        }
-                    }
+                    bts &= ~__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
                 }
-                if (stream_minp) {
-                    lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
-                    if (lane == 0 && lmax > seen_max) { uint32_t old = atomicMax(&s.runmax, lmax); flag = flag || lmax > old; }
+                all |= bts << (u * E::PER_VEC);
+            }
+            const uint32_t cnt = __popc(all);
+            if (__any_sync(0xFFFFFFFFu, cnt != 0)) {
+                // one reservation per warp, then every lane writes its survivors (re-read from the stage)
+                const uint32_t inc = warp_incl_scan_u32(cnt);
+                const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                uint32_t base = 0;
+                if (lane == 31) base = atomicAdd(&s.cand_cnt, total);
+                base = __shfl_sync(0xFFFFFFFFu, base, 31);
+                flag = flag || base + total + 1u >= trig;
+                if (base + total > (uint32_t)CAND_CAP) { if (lane == 31) s.overflow = 1u; flag = true; }
+                else {
+                    uint32_t slot = base + inc - cnt;
+                    uint32_t lmax = 0;
+                    while (all) {
+                        const int pbit = __ffs(all) - 1;
+                        all &= all - 1;
+                        const int u = pbit / E::PER_VEC, e = pbit % E::PER_VEC;
+                        const float x = E::load_plain((const void *)(stage + u * NT), e);
+                        const uint32_t key = key_of(__fmul_rn(x, c.invT));
+                        cs.cand[slot++] = comp_of(key, head + (vbase + u * NT + threadIdx.x) * E::PER_VEC + e);
+                        lmax = key > lmax ? key : lmax;
+                    }
+                    if (stream_minp) {
+                        lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
+                        if (lane == 0 && lmax > seen_max) { uint32_t old = atomicMax(&s.runmax, lmax); flag = flag || lmax > old; }
+                    }
                 }
             }
         }
         const bool need = __syncthreads_or(flag);      // also: every thread is done reading this stage
-        if (threadIdx.x == 0 && tile + rg.nstages < ntiles && !s.timeout) ring_issue(rg, vp, nvec, tile + rg.nstages);
+        if (threadIdx.x == 0 && tile + rg.nstages < ntiles && !s.timeout) ring_issue(rg, vp, nvec, tile + rg.nstages, st);
+        if (++st == rg.nstages) { st = 0; parity ^= 1u; }
         if (need) {
             // every thread is here, so nobody appends until the barriers below are passed
             int n = (int)s.cand_cnt;
@@ -1242,8 +1281,8 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     __syncthreads();
 
     CandSmem cs;
-    cs.cand = (u64 *)smem;                                  // 16 KiB
-    cs.hist = (uint32_t *)(smem + CAND_CAP * 8);            // 8 KiB while selecting ...
+    cs.cand = (u64 *)smem;                                  // 8 KiB
+    cs.hist = (uint32_t *)(smem + CAND_CAP * 8);            // 2 KiB while selecting ...
     cs.sorted = (u64 *)(smem + CAND_CAP * 8);               // ... then the 4 KiB sorted list
     bool done = false;
     if (!(a.flags & ALBIREO_FLAG_FORCE_GENERAL)) done = candidate_path<DT>(s, cs, rg, c, rp, a, b, out);
@@ -1271,7 +1310,7 @@ int ring_stages_for(int V, bool with_history) {
     long fixed = COMMON_BYTES + MAX_STAGES * 8 + (with_history ? (long)history_smem_bytes(V) : 0);
     long n = (budget - fixed) / STAGE_BYTES;
     if (n < 2) n = 2;
-    if (n > 6) n = 6;
+    if (n > 4) n = 4;
     return (int)n;
 }
 size_t smem_bytes_for(int V, bool with_history, int nstages) {
