@@ -136,6 +136,7 @@ struct BlockScratch {
     uint32_t list_cnt;
     uint32_t cand_cnt, overflow, runmax, timeout;
     uint32_t r32a[NWARPS], r32b[NWARPS];
+    uint32_t mm_max, mm_min;
 };
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -642,6 +643,20 @@ __device__ __forceinline__ void ring_issue(const Ring &rg, const uint4 *vp, int 
     mbar_expect_tx(&rg.bar[st], (uint32_t)nv * 16u);
     bulk_g2s(rg.buf + (size_t)st * STAGE_BYTES, vp + v0, (uint32_t)nv * 16u, &rg.bar[st]);
 }
+// Tile 0 arrives in two copies: its first NT vectors (the warm-up slice, one vector per thread) on
+// their own mbarrier so that the threshold can be set up while the rest is still in flight.
+__device__ __forceinline__ void ring_issue_first(const Ring &rg, const uint4 *vp, int nvec) {
+    const int na = nvec < NT ? nvec : NT;
+    int nb = nvec - na; if (nb > NT * (TILE_VECS - 1)) nb = NT * (TILE_VECS - 1);
+    mbar_expect_tx(&rg.bar[MAX_STAGES - 1], (uint32_t)na * 16u);
+    bulk_g2s(rg.buf, vp, (uint32_t)na * 16u, &rg.bar[MAX_STAGES - 1]);
+    if (nb > 0) {
+        mbar_expect_tx(&rg.bar[0], (uint32_t)nb * 16u);
+        bulk_g2s(rg.buf + (size_t)na * 16, vp + na, (uint32_t)nb * 16u, &rg.bar[0]);
+    } else {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rg.bar[0])) : "memory");
+    }
+}
 // waits for the copies of tiles [t0, t1) so that the CTA may leave or reuse the ring
 __device__ void ring_drain(const Ring &rg, int t0, int t1) {
     for (int t = t0; t < t1; ++t) mbar_wait(&rg.bar[t % rg.nstages], (uint32_t)(t / rg.nstages) & 1u);
@@ -689,12 +704,15 @@ __device__ void block_minmax_u32(BlockScratch &s, uint32_t v, uint32_t &mn, uint
 // holds the k-th largest such key.  Returns false if fewer than k keys are in range.
 // On success [lo, hi] is narrowed to that bin and k to the rank inside it; `shift` tells
 // the bin width (0: the bin is a single key, i.e. lo is exactly the k-th largest key).
-__device__ bool cand_select_pass(BlockScratch &s, const CandSmem &cs, int n, uint32_t &k, uint32_t &lo, uint32_t &hi, int &shift) {
+__device__ bool cand_select_pass(BlockScratch &s, const CandSmem &cs, int n, uint32_t &k, uint32_t &lo, uint32_t &hi, int &shift,
+                                 bool zeroed = false) {
     const uint32_t width = hi - lo;
     shift = width < (uint32_t)SEL_BINS ? 0 : (32 - __clz(width)) - 9;
-    cs.hist[threadIdx.x] = 0;
-    if (threadIdx.x == 0) s.found_digit = 0xFFFFFFFFu;
-    __syncthreads();
+    if (!zeroed) {          // (a caller that zeroed the bins and found_digit before its last barrier skips this)
+        cs.hist[threadIdx.x] = 0;
+        if (threadIdx.x == 0) s.found_digit = 0xFFFFFFFFu;
+        __syncthreads();
+    }
     for (int i = threadIdx.x; i < n; i += NT) {
         uint32_t key = (uint32_t)(cs.cand[i] >> 32);
         if (key >= lo && key <= hi) atomicAdd(&cs.hist[(key - lo) >> shift], 1u);
@@ -879,34 +897,34 @@ __device__ __forceinline__ void cand_append_one(BlockScratch &s, u64 *cand, u64 
     if (slot < (uint32_t)CAND_CAP) cand[slot] = C; else s.overflow = 1u;
 }
 
-// Cuts and draw over the sorted candidate list, by one warp (no block barriers).
-// sorted[0..n) best first; efx: scratch for n fixed-point masses.
-__device__ void final_stage_warp(const u64 *sorted, u64 *efx, int n, int L6, bool has_minp, const RowParams &rp,
-                                 const SampleArgs &a, int b, RowOut &out) {
+// Cuts and draw over the sorted candidate list.  Phase 1 (all threads, one candidate each):
+// masses and race scores.  Phase 2 (warp 0): the cuts as prefix operations, the argmax.
+// sorted[0..n) best first; efx / gsc: scratch for n fixed-point masses and race scores.
+__device__ void final_stage(BlockScratch &s, const u64 *sorted, u64 *efx, u64 *gsc, int n, int L6, bool has_minp,
+                            const RowParams &rp, const SampleArgs &a, int b, RowOut &out) {
+    const int j = threadIdx.x;
     const int lane = threadIdx.x & 31;
     const float zmax = unkey((uint32_t)(sorted[0] >> 32));
-    // min-p: a prefix; at least one survivor
-    int L7 = L6;
-    if (has_minp) {
-        const double ln_minp = log((double)rp.min_p);
-        int cnt = 0;
-        for (int j = lane; j < L6; j += 32) {
-            const double dj = (double)unkey((uint32_t)(sorted[j] >> 32)) - (double)zmax;
-            cnt += dj >= ln_minp;
-        }
-        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-        L7 = cnt < 1 ? 1 : cnt;
+    bool in7 = j < L6;
+    if (j < n) {
+        const u64 C = sorted[j];
+        const float z = unkey((uint32_t)(C >> 32));
+        const float d = __fsub_rn(z, zmax);
+        efx[j] = mass_fx(d);
+        const int id = comp_idx(C);
+        const float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, id));
+        gsc[j] = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)id);
+        if (has_minp) in7 = in7 && ((double)z - (double)zmax >= log((double)rp.min_p));
     }
-    // masses in fixed point (integer sums are exact, so the prefix sums are order-independent)
+    // min-p keeps a prefix of the order, at least one element (the barrier also publishes efx / gsc)
+    int L7 = __syncthreads_count(in7);
+    if (L7 < 1) L7 = 1;
+    if (threadIdx.x >= 32) return;
+
+    // masses are fixed point: integer sums are exact, so prefix sums do not depend on the order
     u64 tot = 0;
-    for (int j = lane; j < L7; j += 32) {
-        const float d = __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax);
-        const u64 e = mass_fx(d);
-        efx[j] = e;
-        tot += e;
-    }
+    for (int q = lane; q < L7; q += 32) tot += efx[q];
     tot = warp_sum_u64(tot);
-    __syncwarp();
     int L8 = L7;
     u64 S_fx = tot;
     if (!rp.greedy && rp.top_p < 1.0f) {
@@ -914,62 +932,65 @@ __device__ void final_stage_warp(const u64 *sorted, u64 *efx, int n, int L6, boo
         u64 target = t <= 1.0 ? 1ull : (u64)t;
         if (target > tot) target = tot;
         // smallest prefix whose mass reaches the target
-        u64 carry = 0;
+        u64 carry = 0, kept_mass = 0;
         int keepn = 0;
-        u64 kept_mass = 0;
-        for (int j0 = 0; j0 < L7; j0 += 32) {
-            const int j = j0 + lane;
-            const u64 e = j < L7 ? efx[j] : 0ull;
+        for (int q0 = 0; q0 < L7; q0 += 32) {
+            const int q = q0 + lane;
+            const u64 e = q < L7 ? efx[q] : 0ull;
             u64 inc = e;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t2; }
-            const u64 before = carry + inc - e;
-            const bool keep = j < L7 && before < target;
+            const bool keep = q < L7 && carry + inc - e < target;
             const uint32_t mk = __ballot_sync(0xFFFFFFFFu, keep);
             keepn += __popc(mk);
-            if (mk) {
-                const int last = 31 - __clz(mk);
-                kept_mass = carry + __shfl_sync(0xFFFFFFFFu, inc, last);
-            }
+            if (mk) kept_mass = carry + __shfl_sync(0xFFFFFFFFu, inc, 31 - __clz(mk));
             carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
             if (mk != 0xFFFFFFFFu) break;           // warp-uniform
         }
         L8 = keepn; S_fx = kept_mass;
     }
     const float lnS = logf((float)S_fx * (1.0f / FX_SCALE));
-    // race over the kept prefix
     int tok = comp_idx(sorted[0]);
     float lp_tok = 0.0f;
     if (L8 > 1) {
         u64 best = 0;
-        for (int j = lane; j < L8; j += 32) {
-            const int id = comp_idx(sorted[j]);
-            const float d = __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax);
-            const float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, id));
-            const u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)id);
-            best = G > best ? G : best;
-        }
+        for (int q = lane; q < L8; q += 32) { u64 G = gsc[q]; best = G > best ? G : best; }
         best = warp_max_u64(best);
         tok = comp_idx(best);
-        // logprob of the winner: find it in the list
         float lp = 0.0f; bool mine = false;
-        for (int j = lane; j < L8; j += 32)
-            if (comp_idx(sorted[j]) == tok) { mine = true; lp = __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax) - lnS; }
+        for (int q = lane; q < L8; q += 32)
+            if (comp_idx(sorted[q]) == tok) { mine = true; lp = __fsub_rn(unkey((uint32_t)(sorted[q] >> 32)), zmax) - lnS; }
         const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
         lp_tok = __shfl_sync(0xFFFFFFFFu, lp, __ffs(who) - 1);
     }
     out.token = tok; out.logprob = lp_tok; out.n_keep = L8;
     if (a.num_top > 0) {
-        for (int j = lane; j < a.num_top && j < L8; j += 32) {
-            const int64_t q = (int64_t)b * a.num_top + j;
-            a.out_top_ids[q] = comp_idx(sorted[j]);
-            a.out_top_logprobs[q] = (L8 == 1) ? 0.0f : __fsub_rn(unkey((uint32_t)(sorted[j] >> 32)), zmax) - lnS;
+        for (int q = lane; q < a.num_top && q < L8; q += 32) {
+            const int64_t o = (int64_t)b * a.num_top + q;
+            a.out_top_ids[o] = comp_idx(sorted[q]);
+            a.out_top_logprobs[o] = (L8 == 1) ? 0.0f : __fsub_rn(unkey((uint32_t)(sorted[q] >> 32)), zmax) - lnS;
         }
     }
 }
 
+// Sorts cand[0..n) (all distinct, n <= SORT_MAX) into sorted[], best first, by rank counting;
+// several threads share the comparisons of one element when n is small.
+__device__ void rank_sort(const u64 *cand, u64 *sorted, int n) {
+    int parts = 1;
+    while (parts < 8 && n * parts * 2 <= NT) parts *= 2;
+    const int j = threadIdx.x / parts, part = threadIdx.x % parts;
+    u64 C = 0;
+    int rank = 0;
+    if (j < n) {
+        C = cand[j];
+        for (int q = part; q < n; q += parts) rank += cand[q] > C;
+    }
+    for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+    if (j < n && part == 0) sorted[rank] = C;
+}
+
 // Returns false if the row must be handled by the general path instead.  On success the
-// results are in `out` for warp 0 only (the other warps return early).
+// results are in `out` for warp 0 only.
 template <int DT>
 __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &rg, const RowCtx &c,
                                const RowParams &rp, const SampleArgs &a, int b, RowOut &out) {
@@ -985,6 +1006,11 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     // top-k stage's set is known exactly
     const bool stream_minp = has_minp && !(has_topk && a.dbg_topk_ids != nullptr);
     const int lane = threadIdx.x & 31;
+    // Thread -> vector map inside each group of NT vectors: lane l of warp w takes vector
+    // 16 l + ((w + l) & 15).  Consecutive vectors land in different warps (the head of the
+    // vocabulary, where large logits cluster, is shared by all warps) and the 16-byte shared
+    // memory reads of a quarter warp still fall in distinct bank groups.
+    const int pvec = 16 * lane + (((threadIdx.x >> 5) + lane) & 15);
 
     const uintptr_t addr = (uintptr_t)c.row;
     int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
@@ -995,12 +1021,16 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
 
     if (threadIdx.x == 0) {
         s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
+        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu;
         for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
+        mbar_init(&rg.bar[MAX_STAGES - 1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (ntiles > 0) ring_issue_first(rg, vp, nvec);
         const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
-        for (int t = 0; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
+        for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
     }
+    cs.hist[threadIdx.x] = 0;
     __syncthreads();
 
     uint32_t tau_key = KEY_MIN_FINITE;
@@ -1009,13 +1039,49 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     const uint32_t trig0 = has_topk ? (uint32_t)min(CAND_CAP / 2, 4 * k + 64) : (uint32_t)(CAND_CAP / 2);
     uint32_t trig = trig0;
 
+    if (ntiles > 0) {
+        // warm-up on the first NT vectors: the k-th largest of the per-thread maxima (each an
+        // unpenalised element of the row, all distinct) is a lower bound of the row's k-th
+        // largest score
+        bool bad = !mbar_wait(&rg.bar[MAX_STAGES - 1], 0);
+        uint32_t mk = 0;
+        if (pvec < nvec && !bad) {
+            const uint4 q = ((const uint4 *)rg.buf)[pvec];
+            const int i0 = head + pvec * E::PER_VEC;
+            if (c.has_hist && (__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u)))
+                mk = masked_vmax_key<DT>(c, q, i0);
+            else
+                mk = T::vmax_key(q, c.invT);
+        }
+        if (mk < KEY_MIN_FINITE || mk >= KEY_POS_INF) mk = 0;
+        cs.cand[threadIdx.x] = (u64)mk << 32;
+        {
+            const uint32_t wmx = __reduce_max_sync(0xFFFFFFFFu, mk);
+            const uint32_t wmn = __reduce_min_sync(0xFFFFFFFFu, mk ? mk : 0xFFFFFFFFu);
+            if (lane == 0 && wmx) { atomicMax(&s.mm_max, wmx); atomicMin(&s.mm_min, wmn); }
+        }
+        if (bad) s.timeout = 1u;
+        __syncthreads();
+        const uint32_t kmax = s.mm_max, kmin = s.mm_min;
+        if (stream_minp && threadIdx.x == 0) s.runmax = kmax;
+        // fewer than k valid maxima: the select fails and tau stays at its floor
+        if (has_topk && kmax) {
+            uint32_t kk = (uint32_t)k, lo = kmin, hi = kmax; int shift;
+            if (cand_select_pass(s, cs, NT, kk, lo, hi, shift, true)) tau_key = lo;
+        }
+        if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
+        seen_max = kmax;
+        thr = T::raw_threshold(tau_key, c.invT);
+        if (!(has_topk && kmax)) __syncthreads();       // (the select ends with a barrier of its own)
+    }
+
     int st = 0;                      // ring stage of the current tile
     uint32_t parity = 0;             // its mbarrier phase
     for (int tile = 0; tile < ntiles; ++tile) {
         const int vbase = tile * NT * TILE_VECS;
-        bool flag = false;
+        bool flag = (tile == 0) && s.timeout != 0u;      // the warm-up slice never arrived
         if (!mbar_wait(&rg.bar[st], parity)) { s.timeout = 1u; flag = true; }
-        const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + threadIdx.x;
+        const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + pvec;
         uint4 cur[TILE_VECS];
         if (vbase + NT * TILE_VECS <= nvec && !flag) {
 #pragma unroll
@@ -1023,39 +1089,10 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         } else {
 #pragma unroll
             for (int u = 0; u < TILE_VECS; ++u)
-                cur[u] = (vbase + u * NT + (int)threadIdx.x < nvec && !flag) ? stage[u * NT] : T::fill();
+                cur[u] = (vbase + u * NT + pvec < nvec && !flag) ? stage[u * NT] : T::fill();
         }
-        if (tile == 0) {
-            // warm-up: the k-th largest of the per-thread maxima (each an unpenalised element of
-            // the row, all distinct) is a lower bound of the row's k-th largest score
-            uint32_t mk = 0;
-#pragma unroll
-            for (int u = 0; u < TILE_VECS; ++u) {
-                const int v = u * NT + threadIdx.x;
-                if (v < nvec) {
-                    const int i0 = head + v * E::PER_VEC;
-                    uint32_t kk;
-                    if (c.has_hist && (__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u)))
-                        kk = masked_vmax_key<DT>(c, cur[u], i0);
-                    else
-                        kk = T::vmax_key(cur[u], c.invT);
-                    mk = kk > mk ? kk : mk;
-                }
-            }
-            if (mk < KEY_MIN_FINITE || mk >= KEY_POS_INF) mk = 0;
-            cs.cand[threadIdx.x] = (u64)mk << 32;
-            const int valid = __syncthreads_count(mk != 0);
-            uint32_t kmin, kmax;
-            block_minmax_u32(s, mk, kmin, kmax);
-            if (stream_minp && threadIdx.x == 0) s.runmax = kmax;
-            if (has_topk && valid >= k) tau_key = cand_select_approx(s, cs, NT, k, kmin, kmax);
-            if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
-            seen_max = kmax;
-            thr = T::raw_threshold(tau_key, c.invT);
-            __syncthreads();
-        }
-        // scan: one cheap test for the whole tile share of this thread; the exact element test
-        // only in warps where some vector may pass
+        // scan: one cheap test for this thread's share of the tile; the element test only in
+        // warps where some vector may pass
         if (__any_sync(0xFFFFFFFFu, T::any_may_pass(cur, thr, c.invT))) {
             // per-element test in the test domain (a superset of key >= tau), minus penalised tokens
             uint32_t all = 0;
@@ -1063,7 +1100,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             for (int u = 0; u < TILE_VECS; ++u) {
                 uint32_t bts = T::elem_bits(cur[u], thr, c.invT);
                 if (c.has_hist && bts) {
-                    const int i0 = head + (vbase + u * NT + threadIdx.x) * E::PER_VEC;
+                    const int i0 = head + (vbase + u * NT + pvec) * E::PER_VEC;
                     bts &= ~__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
                 }
                 all |= bts << (u * E::PER_VEC);
@@ -1087,7 +1124,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
                         const int u = pbit / E::PER_VEC, e = pbit % E::PER_VEC;
                         const float x = E::load_plain((const void *)(stage + u * NT), e);
                         const uint32_t key = key_of(__fmul_rn(x, c.invT));
-                        cs.cand[slot++] = comp_of(key, head + (vbase + u * NT + threadIdx.x) * E::PER_VEC + e);
+                        cs.cand[slot++] = comp_of(key, head + (vbase + u * NT + pvec) * E::PER_VEC + e);
                         lmax = key > lmax ? key : lmax;
                     }
                     if (stream_minp) {
@@ -1192,13 +1229,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     }
     if (n > SORT_MAX || n < 1) return false;
 
-    // sort by rank counting (all composites distinct); `sorted` reuses the histogram memory
-    if (threadIdx.x < n) {
-        const u64 C = cs.cand[threadIdx.x];
-        int rank = 0;
-        for (int j = 0; j < n; ++j) rank += cs.cand[j] > C;
-        cs.sorted[rank] = C;
-    }
+    // `sorted` reuses the select bins
+    rank_sort(cs.cand, cs.sorted, n);
     const int L6 = has_topk ? (n < k ? n : k) : n;
     int n_topk = L6;
     if (!topk_exact_known && a.out_num_topk) {
@@ -1212,7 +1244,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     out.n_topk = n_topk;
     if (a.dbg_topk_ids && has_topk && L6 <= a.dbg_cap && threadIdx.x < L6)
         a.dbg_topk_ids[(int64_t)b * a.dbg_cap + threadIdx.x] = comp_idx(cs.sorted[threadIdx.x]);
-    if (threadIdx.x < 32) final_stage_warp(cs.sorted, cs.cand, n, L6, has_minp, rp, a, b, out);
+    final_stage(s, cs.sorted, cs.cand, cs.cand + SORT_MAX, n, L6, has_minp, rp, a, b, out);
     return true;
 }
 
