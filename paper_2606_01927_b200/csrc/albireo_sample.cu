@@ -43,7 +43,7 @@ constexpr int TILE_VECS = 4;            // 16-byte vectors per thread per tile
 constexpr int STAGE_BYTES = NT * TILE_VECS * 16;   // one ring stage = one tile (32 KiB)
 constexpr int MAX_STAGES = 8;
 constexpr int WAIT_CAP = 1 << 20;       // mbarrier polls before a wait gives up
-constexpr int COMMON_BYTES = 12288;     // candidate list (8 KiB) + select bins / sorted list (4 KiB)
+constexpr int COMMON_BYTES = 10240;     // candidate composites (8 KiB) + select bins (2 KiB)
 constexpr uint32_t KEY_MIN_FINITE = 0x00800000u;   // key(-FLT_MAX); key(-inf) is one below
 constexpr uint32_t KEY_POS_INF = 0xFF800000u;      // key(+inf)
 constexpr float FX_SCALE = 1099511627776.0f;       // 2^40: fixed-point scale of masses
@@ -137,6 +137,9 @@ struct BlockScratch {
     uint32_t cand_cnt, overflow, runmax, timeout;
     uint32_t r32a[NWARPS], r32b[NWARPS];
     uint32_t mm_max, mm_min;
+    uint32_t done[MAX_STAGES];   // warps finished with each ring stage
+    uint32_t maint_at;           // tile index before which every warp meets (0xFFFFFFFF: none)
+    uint32_t issued;             // tiles whose copy has been issued so far
 };
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -673,9 +676,10 @@ __device__ void ring_drain(const Ring &rg, int t0, int t1) {
 // they are evaluated from the history bitmap after the stream.
 
 struct CandSmem {
-    u64 *cand;        // CAND_CAP composites; after the sort: fixed-point masses of the sorted list
-    uint32_t *hist;   // SEL_BINS bins while selecting ...
-    u64 *sorted;      // ... SORT_MAX composites (best first) afterwards: same memory
+    u64 *cand;        // CAND_CAP composites
+    uint32_t *hist;   // SEL_BINS bins while selecting
+    // scratch of the final stage, in the (by then idle) ring: sorted composites, masses, race scores
+    u64 *sorted, *efx, *gsc;
 };
 
 constexpr int SEL_BINS = NT;            // one bin per thread
@@ -888,80 +892,93 @@ __device__ __noinline__ uint32_t masked_vmax_key(const RowCtx &c, uint4 q, int i
 }
 
 // Single appends outside the streaming loop (scalar head/tail, penalised tokens).
-__device__ __forceinline__ void cand_append_one(BlockScratch &s, u64 *cand, u64 C) {
+__device__ __forceinline__ void cand_append_one(BlockScratch &s, const CandSmem &cs, u64 C) {
     cg::coalesced_group g = cg::coalesced_threads();
     uint32_t base = 0;
     if (g.thread_rank() == 0) base = atomicAdd(&s.cand_cnt, g.size());
     base = g.shfl(base, 0);
     const uint32_t slot = base + g.thread_rank();
-    if (slot < (uint32_t)CAND_CAP) cand[slot] = C; else s.overflow = 1u;
+    if (slot < (uint32_t)CAND_CAP) cs.cand[slot] = C; else s.overflow = 1u;
+    atomicMax(&s.runmax, (uint32_t)(C >> 32));
 }
 
-// Cuts and draw over the sorted candidate list.  Phase 1 (all threads, one candidate each):
-// masses and race scores.  Phase 2 (warp 0): the cuts as prefix operations, the argmax.
-// sorted[0..n) best first; efx / gsc: scratch for n fixed-point masses and race scores.
-__device__ void final_stage(BlockScratch &s, const u64 *sorted, u64 *efx, u64 *gsc, int n, int L6, bool has_minp,
+// Final stage over the candidate list cand[0..n) (all distinct, n <= SORT_MAX), whose largest
+// score is zmax.  Step 1 (all threads): each candidate's rank by counting (several threads share
+// the comparisons of one candidate when n is small), its mass and its race score, written to its
+// sorted position.  Step 2 (warp 0): the cuts as prefix operations and the argmax of the race.
+__device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, float zmax, bool has_minp,
                             const RowParams &rp, const SampleArgs &a, int b, RowOut &out) {
-    const int j = threadIdx.x;
     const int lane = threadIdx.x & 31;
-    const float zmax = unkey((uint32_t)(sorted[0] >> 32));
-    bool in7 = j < L6;
+    int parts = 1;
+    while (parts < 8 && n * parts * 2 <= NT) parts *= 2;
+    const int j = threadIdx.x / parts, part = threadIdx.x % parts;
+    u64 C = 0;
+    int rank = 0;
+    float g = 0.0f;
     if (j < n) {
-        const u64 C = sorted[j];
+        C = cs.cand[j];
+        if (part == 0) g = neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, comp_idx(C)));
+        for (int q = part; q < n; q += parts) rank += cs.cand[q] > C;
+    }
+    for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+    bool in7 = false;
+    if (j < n && part == 0) {
         const float z = unkey((uint32_t)(C >> 32));
         const float d = __fsub_rn(z, zmax);
-        efx[j] = mass_fx(d);
-        const int id = comp_idx(C);
-        const float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, id));
-        gsc[j] = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)id);
-        if (has_minp) in7 = in7 && ((double)z - (double)zmax >= log((double)rp.min_p));
+        cs.sorted[rank] = C;
+        cs.efx[rank] = mass_fx(d);
+        cs.gsc[rank] = ((u64)orderable_f32(d + g) << 32) | (uint32_t)C;
+        in7 = rank < L6 && (!has_minp || ((double)z - (double)zmax >= log((double)rp.min_p)));
     }
-    // min-p keeps a prefix of the order, at least one element (the barrier also publishes efx / gsc)
+    // min-p keeps a prefix of the order, at least one element (the barrier also publishes step 1)
     int L7 = __syncthreads_count(in7);
     if (L7 < 1) L7 = 1;
+    if (a.dbg_topk_ids && L6 <= a.dbg_cap && (int)threadIdx.x < L6 && (rp.greedy || (rp.top_k >= 1 && rp.top_k < a.V)))
+        a.dbg_topk_ids[(int64_t)b * a.dbg_cap + threadIdx.x] = comp_idx(cs.sorted[threadIdx.x]);
     if (threadIdx.x >= 32) return;
 
-    // masses are fixed point: integer sums are exact, so prefix sums do not depend on the order
-    u64 tot = 0;
-    for (int q = lane; q < L7; q += 32) tot += efx[q];
-    tot = warp_sum_u64(tot);
+    const u64 *sorted = cs.sorted, *gsc = cs.gsc;
+    u64 *efx = cs.efx;
+    // Masses are fixed point: integer sums are exact, so the prefix sums do not depend on the
+    // order of the additions.  Inclusive prefix sums replace the masses in place.
+    u64 carry = 0;
+    for (int q0 = 0; q0 < L7; q0 += 32) {
+        const int q = q0 + lane;
+        u64 inc = q < L7 ? efx[q] : 0ull;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t2; }
+        inc += carry;
+        if (q < L7) efx[q] = inc;
+        carry = __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
+    const u64 tot = carry;
     int L8 = L7;
     u64 S_fx = tot;
     if (!rp.greedy && rp.top_p < 1.0f) {
         double t = ceil((double)rp.top_p * (double)tot);
         u64 target = t <= 1.0 ? 1ull : (u64)t;
         if (target > tot) target = tot;
-        // smallest prefix whose mass reaches the target
-        u64 carry = 0, kept_mass = 0;
-        int keepn = 0;
-        for (int q0 = 0; q0 < L7; q0 += 32) {
-            const int q = q0 + lane;
-            const u64 e = q < L7 ? efx[q] : 0ull;
-            u64 inc = e;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t2; }
-            const bool keep = q < L7 && carry + inc - e < target;
-            const uint32_t mk = __ballot_sync(0xFFFFFFFFu, keep);
-            keepn += __popc(mk);
-            if (mk) kept_mass = carry + __shfl_sync(0xFFFFFFFFu, inc, 31 - __clz(mk));
-            carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
-            if (mk != 0xFFFFFFFFu) break;           // warp-uniform
-        }
-        L8 = keepn; S_fx = kept_mass;
+        __syncwarp();
+        // smallest prefix whose mass reaches the target: count the elements whose inclusive sum is below it
+        int below = 0;
+        for (int q = lane; q < L7; q += 32) below += efx[q] < target;
+        below = __reduce_add_sync(0xFFFFFFFFu, below);
+        L8 = below + 1 < L7 ? below + 1 : L7;
+        S_fx = efx[L8 - 1];
     }
     const float lnS = logf((float)S_fx * (1.0f / FX_SCALE));
     int tok = comp_idx(sorted[0]);
     float lp_tok = 0.0f;
     if (L8 > 1) {
-        u64 best = 0;
-        for (int q = lane; q < L8; q += 32) { u64 G = gsc[q]; best = G > best ? G : best; }
-        best = warp_max_u64(best);
-        tok = comp_idx(best);
-        float lp = 0.0f; bool mine = false;
-        for (int q = lane; q < L8; q += 32)
-            if (comp_idx(sorted[q]) == tok) { mine = true; lp = __fsub_rn(unkey((uint32_t)(sorted[q] >> 32)), zmax) - lnS; }
-        const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
-        lp_tok = __shfl_sync(0xFFFFFFFFu, lp, __ffs(who) - 1);
+        // argmax of the race score over the kept prefix (ties: lowest id, via the low word ~id)
+        u64 best = 0; int bestq = 0;
+        for (int q = lane; q < L8; q += 32) { u64 G = gsc[q]; if (G > best) { best = G; bestq = q; } }
+        const uint32_t ghi = __reduce_max_sync(0xFFFFFFFFu, (uint32_t)(best >> 32));
+        const uint32_t glo = __reduce_max_sync(0xFFFFFFFFu, (uint32_t)(best >> 32) == ghi ? (uint32_t)best : 0u);
+        const uint32_t who = __ballot_sync(0xFFFFFFFFu, (uint32_t)(best >> 32) == ghi && (uint32_t)best == glo);
+        const int wq = __shfl_sync(0xFFFFFFFFu, bestq, __ffs(who) - 1);
+        tok = comp_idx(sorted[wq]);
+        lp_tok = __fsub_rn(unkey((uint32_t)(sorted[wq] >> 32)), zmax) - lnS;
     }
     out.token = tok; out.logprob = lp_tok; out.n_keep = L8;
     if (a.num_top > 0) {
@@ -971,22 +988,6 @@ __device__ void final_stage(BlockScratch &s, const u64 *sorted, u64 *efx, u64 *g
             a.out_top_logprobs[o] = (L8 == 1) ? 0.0f : __fsub_rn(unkey((uint32_t)(sorted[q] >> 32)), zmax) - lnS;
         }
     }
-}
-
-// Sorts cand[0..n) (all distinct, n <= SORT_MAX) into sorted[], best first, by rank counting;
-// several threads share the comparisons of one element when n is small.
-__device__ void rank_sort(const u64 *cand, u64 *sorted, int n) {
-    int parts = 1;
-    while (parts < 8 && n * parts * 2 <= NT) parts *= 2;
-    const int j = threadIdx.x / parts, part = threadIdx.x % parts;
-    u64 C = 0;
-    int rank = 0;
-    if (j < n) {
-        C = cand[j];
-        for (int q = part; q < n; q += parts) rank += cand[q] > C;
-    }
-    for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
-    if (j < n && part == 0) sorted[rank] = C;
 }
 
 // Returns false if the row must be handled by the general path instead.  On success the
@@ -1021,7 +1022,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
 
     if (threadIdx.x == 0) {
         s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
-        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu;
+        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
+        for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
         for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
         mbar_init(&rg.bar[MAX_STAGES - 1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1029,6 +1031,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         if (ntiles > 0) ring_issue_first(rg, vp, nvec);
         const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
         for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
+        s.issued = (uint32_t)npre;
     }
     cs.hist[threadIdx.x] = 0;
     __syncthreads();
@@ -1075,76 +1078,23 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         if (!(has_topk && kmax)) __syncthreads();       // (the select ends with a barrier of its own)
     }
 
+    // The consumer warps run decoupled: no block barrier per tile.  A stage is refilled by the
+    // last warp that finishes with it.  Block-wide work on the candidate list (tightening the
+    // threshold, overflow, expired waits) happens at a rendezvous: a warp working on tile t asks
+    // for one before tile t + nstages + 1.  No warp can have looked at that boundary yet: it is
+    // reached only after tile t + nstages, whose data is requested only when every warp is done
+    // with tile t.  Every warp checks s.maint_at before each tile.
     int st = 0;                      // ring stage of the current tile
     uint32_t parity = 0;             // its mbarrier phase
     for (int tile = 0; tile < ntiles; ++tile) {
-        const int vbase = tile * NT * TILE_VECS;
-        bool flag = (tile == 0) && s.timeout != 0u;      // the warm-up slice never arrived
-        if (!mbar_wait(&rg.bar[st], parity)) { s.timeout = 1u; flag = true; }
-        const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + pvec;
-        uint4 cur[TILE_VECS];
-        if (vbase + NT * TILE_VECS <= nvec && !flag) {
-#pragma unroll
-            for (int u = 0; u < TILE_VECS; ++u) cur[u] = stage[u * NT];
-        } else {
-#pragma unroll
-            for (int u = 0; u < TILE_VECS; ++u)
-                cur[u] = (vbase + u * NT + pvec < nvec && !flag) ? stage[u * NT] : T::fill();
-        }
-        // scan: one cheap test for this thread's share of the tile; the element test only in
-        // warps where some vector may pass
-        if (__any_sync(0xFFFFFFFFu, T::any_may_pass(cur, thr, c.invT))) {
-            // per-element test in the test domain (a superset of key >= tau), minus penalised tokens
-            uint32_t all = 0;
-#pragma unroll
-            for (int u = 0; u < TILE_VECS; ++u) {
-                uint32_t bts = T::elem_bits(cur[u], thr, c.invT);
-                if (c.has_hist && bts) {
-                    const int i0 = head + (vbase + u * NT + pvec) * E::PER_VEC;
-                    bts &= ~__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
-                }
-                all |= bts << (u * E::PER_VEC);
-            }
-            const uint32_t cnt = __popc(all);
-            if (__any_sync(0xFFFFFFFFu, cnt != 0)) {
-                // one reservation per warp, then every lane writes its survivors (re-read from the stage)
-                const uint32_t inc = warp_incl_scan_u32(cnt);
-                const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
-                uint32_t base = 0;
-                if (lane == 31) base = atomicAdd(&s.cand_cnt, total);
-                base = __shfl_sync(0xFFFFFFFFu, base, 31);
-                flag = flag || base + total + 1u >= trig;
-                if (base + total > (uint32_t)CAND_CAP) { if (lane == 31) s.overflow = 1u; flag = true; }
-                else {
-                    uint32_t slot = base + inc - cnt;
-                    uint32_t lmax = 0;
-                    while (all) {
-                        const int pbit = __ffs(all) - 1;
-                        all &= all - 1;
-                        const int u = pbit / E::PER_VEC, e = pbit % E::PER_VEC;
-                        const float x = E::load_plain((const void *)(stage + u * NT), e);
-                        const uint32_t key = key_of(__fmul_rn(x, c.invT));
-                        cs.cand[slot++] = comp_of(key, head + (vbase + u * NT + pvec) * E::PER_VEC + e);
-                        lmax = key > lmax ? key : lmax;
-                    }
-                    if (stream_minp) {
-                        lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
-                        if (lane == 0 && lmax > seen_max) { uint32_t old = atomicMax(&s.runmax, lmax); flag = flag || lmax > old; }
-                    }
-                }
-            }
-        }
-        const bool need = __syncthreads_or(flag);      // also: every thread is done reading this stage
-        if (threadIdx.x == 0 && tile + rg.nstages < ntiles && !s.timeout) ring_issue(rg, vp, nvec, tile + rg.nstages, st);
-        if (++st == rg.nstages) { st = 0; parity ^= 1u; }
-        if (need) {
-            // every thread is here, so nobody appends until the barriers below are passed
+        if ((uint32_t)tile == *(volatile uint32_t *)&s.maint_at) {
+            __syncthreads();                       // every warp is between tiles: nobody appends
             int n = (int)s.cand_cnt;
             const uint32_t ovf = s.overflow, rmax = s.runmax, tmo = s.timeout;
             __syncthreads();
+            if (threadIdx.x == 0) s.maint_at = 0xFFFFFFFFu;
             if (ovf || tmo) {
-                const int issued = min(ntiles, tile + 1 + rg.nstages);
-                ring_drain(rg, tmo ? tile : tile + 1, tmo ? min(ntiles, tile + rg.nstages) : issued);   // after a timeout nothing new was issued
+                ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
                 if (tmo) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; return true; }
                 __syncthreads();
                 return false;
@@ -1169,7 +1119,93 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
                 if (trig < trig0) trig = trig0;
             }
             if (changed) thr = T::raw_threshold(tau_key, c.invT);
+            __syncthreads();                       // s.maint_at is reset before anyone asks again
         }
+        const int vbase = tile * NT * TILE_VECS;
+        bool ask = false;                          // ask for a rendezvous
+        const bool dead = *(volatile uint32_t *)&s.timeout != 0u;   // a wait expired somewhere: only keep the protocol going
+        if (!dead) {
+            if (!mbar_wait(&rg.bar[st], parity)) { s.timeout = 1u; ask = true; }
+            else {
+                const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + pvec;
+                uint4 cur[TILE_VECS];
+                if (vbase + NT * TILE_VECS <= nvec) {
+#pragma unroll
+                    for (int u = 0; u < TILE_VECS; ++u) cur[u] = stage[u * NT];
+                } else {
+#pragma unroll
+                    for (int u = 0; u < TILE_VECS; ++u)
+                        cur[u] = (vbase + u * NT + pvec < nvec) ? stage[u * NT] : T::fill();
+                }
+                // scan: one cheap test for this thread's share of the tile; the element test only in
+                // warps where some vector may pass
+                if (__any_sync(0xFFFFFFFFu, T::any_may_pass(cur, thr, c.invT))) {
+                    // per-element test in the test domain (a superset of key >= tau), minus penalised tokens
+                    uint32_t all = 0;
+#pragma unroll
+                    for (int u = 0; u < TILE_VECS; ++u) {
+                        uint32_t bts = T::elem_bits(cur[u], thr, c.invT);
+                        if (c.has_hist && bts) {
+                            const int i0 = head + (vbase + u * NT + pvec) * E::PER_VEC;
+                            bts &= ~__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+                        }
+                        all |= bts << (u * E::PER_VEC);
+                    }
+                    const uint32_t cnt = __popc(all);
+                    if (__any_sync(0xFFFFFFFFu, cnt != 0)) {
+                        // one reservation per warp, then every lane writes its survivors (re-read from the stage)
+                        const uint32_t inc = warp_incl_scan_u32(cnt);
+                        const uint32_t total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                        uint32_t base = 0;
+                        if (lane == 31) base = atomicAdd(&s.cand_cnt, total);
+                        base = __shfl_sync(0xFFFFFFFFu, base, 31);
+                        ask = base + total + 1u >= trig;
+                        if (base + total > (uint32_t)CAND_CAP) { if (lane == 31) s.overflow = 1u; ask = true; }
+                        else {
+                            uint32_t slot = base + inc - cnt;
+                            uint32_t lmax = 0;
+                            while (all) {
+                                const int pbit = __ffs(all) - 1;
+                                all &= all - 1;
+                                const int u = pbit / E::PER_VEC, e = pbit % E::PER_VEC;
+                                const float x = E::load_plain((const void *)(stage + u * NT), e);
+                                const uint32_t key = key_of(__fmul_rn(x, c.invT));
+                                cs.cand[slot++] = comp_of(key, head + (vbase + u * NT + pvec) * E::PER_VEC + e);
+                                lmax = key > lmax ? key : lmax;
+                            }
+                            lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
+                            if (lane == 0 && lmax > *(volatile uint32_t *)&s.runmax) {
+                                const uint32_t old = atomicMax(&s.runmax, lmax);
+                                ask = ask || (stream_minp && lmax > old && lmax > seen_max);
+                            }
+
+                        }
+                    }
+                }
+            }
+        }
+        if (__any_sync(0xFFFFFFFFu, ask) && lane == 0) atomicMin(&s.maint_at, (uint32_t)(tile + rg.nstages + 1));
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence_block();                 // this warp's reads of the stage come before its arrival
+            const uint32_t old = atomicAdd(&s.done[st], 1u);
+            if (old == (uint32_t)(NWARPS - 1)) {   // last warp done with this stage: refill it
+                s.done[st] = 0;
+                __threadfence_block();
+                if (tile + rg.nstages < ntiles && *(volatile uint32_t *)&s.timeout == 0u) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    ring_issue(rg, vp, nvec, tile + rg.nstages, st);
+                    atomicMax(&s.issued, (uint32_t)(tile + rg.nstages + 1));
+                }
+            }
+        }
+        if (++st == rg.nstages) { st = 0; parity ^= 1u; }
+    }
+    __syncthreads();
+    if (s.timeout) {
+        ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
+        out.status |= ALBIREO_ROW_TIMEOUT; out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0;
+        return true;
     }
     // scalar head and tail of a row that is not 16-byte aligned / not a whole number of vectors
     {
@@ -1179,7 +1215,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             int i = q < head ? q : tail0 + (q - head);
             if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
             uint32_t key = key_of(__fmul_rn(E::load(c.row, i), c.invT));
-            if (key >= tau_key) cand_append_one(s, cs.cand, comp_of(key, i));
+            if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
         }
     }
     // penalised tokens, straight from the history bitmap
@@ -1200,7 +1236,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
                 av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cntv)));
                 av = __fsub_rn(av, c.p);
                 uint32_t key = key_of(__fmul_rn(av, c.invT));
-                if (key >= tau_key) cand_append_one(s, cs.cand, comp_of(key, i));
+                if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
             }
         }
     }
@@ -1210,27 +1246,20 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     __syncthreads();
     if (ovf || n < 1) return false;
 
+    const uint32_t kmax = s.runmax;    // the row's largest score is always a candidate
     bool topk_exact_known = true;      // is min(k, #finite) known without counting?
     if (has_topk) {
         if (n > SORT_MAX || n > 2 * k + 96) {
-            uint32_t lmx = 0, mn, hi;
-            for (int i = threadIdx.x; i < n; i += NT) { uint32_t kk = (uint32_t)(cs.cand[i] >> 32); lmx = kk > lmx ? kk : lmx; }
-            block_minmax_u32(s, lmx, mn, hi);
-            uint32_t t = cand_select_exact(s, cs, n, k, tau_key, hi);
+            uint32_t t = cand_select_exact(s, cs, n, k, tau_key, kmax);
             n = cand_compact(s, cs, n, t);
         }
         if (n < k && stream_minp) topk_exact_known = false;
     } else {
-        uint32_t lmx = 0, mn, hi;
-        for (int i = threadIdx.x; i < n; i += NT) { uint32_t kk = (uint32_t)(cs.cand[i] >> 32); lmx = kk > lmx ? kk : lmx; }
-        block_minmax_u32(s, lmx, mn, hi);
-        n = cand_compact(s, cs, n, minp_key(unkey(hi), rp.min_p));
+        n = cand_compact(s, cs, n, minp_key(unkey(kmax), rp.min_p));
         topk_exact_known = false;
     }
     if (n > SORT_MAX || n < 1) return false;
 
-    // `sorted` reuses the select bins
-    rank_sort(cs.cand, cs.sorted, n);
     const int L6 = has_topk ? (n < k ? n : k) : n;
     int n_topk = L6;
     if (!topk_exact_known && a.out_num_topk) {
@@ -1240,18 +1269,16 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         u64 nfin = block_sum_u64(s, local);
         n_topk = has_topk ? (int)(nfin < (u64)k ? nfin : (u64)k) : (int)nfin;
     }
-    __syncthreads();
     out.n_topk = n_topk;
-    if (a.dbg_topk_ids && has_topk && L6 <= a.dbg_cap && threadIdx.x < L6)
-        a.dbg_topk_ids[(int64_t)b * a.dbg_cap + threadIdx.x] = comp_idx(cs.sorted[threadIdx.x]);
-    final_stage(s, cs.sorted, cs.cand, cs.cand + SORT_MAX, n, L6, has_minp, rp, a, b, out);
+    final_stage(s, cs, n, L6, unkey(kmax), has_minp, rp, a, b, out);
     return true;
 }
 
 // ------------------------------------------------------------------ the kernel
 
-// dynamic shared memory layout (bytes): [24 KiB shared by the two paths: histograms (cnt 8 KiB, mass
-// 16 KiB) or candidates (16 KiB) + 2048 bins / sorted list (8 KiB)][bitmap][coarse][counts]
+// dynamic shared memory layout (bytes): [candidates (8 KiB) + 512 select bins (2 KiB)]
+// [ring: nstages x 32 KiB][mbarriers][bitmap][coarse][counts]; the general path lays its histograms
+// (cnt 8 KiB, mass 16 KiB) over the first 24 KiB, which it may do because the ring is idle by then
 template <int DT>
 __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -1314,8 +1341,10 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
 
     CandSmem cs;
     cs.cand = (u64 *)smem;                                  // 8 KiB
-    cs.hist = (uint32_t *)(smem + CAND_CAP * 8);            // 2 KiB while selecting ...
-    cs.sorted = (u64 *)(smem + CAND_CAP * 8);               // ... then the 4 KiB sorted list
+    cs.hist = (uint32_t *)(smem + CAND_CAP * 8);            // 2 KiB
+    cs.sorted = (u64 *)rg.buf;                              // 3 x 4 KiB in the ring, used after the stream
+    cs.efx = cs.sorted + SORT_MAX;
+    cs.gsc = cs.efx + SORT_MAX;
     bool done = false;
     if (!(a.flags & ALBIREO_FLAG_FORCE_GENERAL)) done = candidate_path<DT>(s, cs, rg, c, rp, a, b, out);
     if (!done) {
