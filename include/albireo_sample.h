@@ -184,6 +184,53 @@ const char *albireo_last_error(const albireo_sampler_t *h);
 /* Number of kernel launches albireo_sample has enqueued through this handle so far. */
 uint64_t albireo_sample_launch_count(const albireo_sampler_t *h);
 
+/* largest history_total albireo_sample_fixed_scratch accepts (entries of its fixed scratch array) */
+#define ALBIREO_FIXED_MAX_HISTORY (1 << 20)
+
+/*
+ * albireo_sample for callers that cannot allocate device memory (the paper has no
+ * counterpart: this entry point exists for integration, not for the method).
+ *
+ * Who needs it: code that gets control when every byte of device memory has already been
+ * handed to someone else's pool, code that must not call cudaMalloc because that would
+ * stall the GPU work around it, and code under a "no allocation after start-up" rule.
+ * Such a caller has nowhere to take the workspace of albireo_sample_init from.  Here the
+ * one piece of scratch the sampler needs -- the per-row history occurrence counts of rows
+ * whose history has more distinct ids than fit on chip -- is a fixed array of
+ * ALBIREO_FIXED_MAX_HISTORY 32-bit counters (4 MiB) inside the library's device image;
+ * every GPU that loads the library holds that array until the process exits.  There is
+ * no handle and no workspace; the entry point calls no allocation routine of any kind.
+ *
+ * Arguments are those of albireo_sample (device pointers, same meaning and layout),
+ * plus history_total = history_offsets[B] as the host knows it (0 without history).
+ * Limits: history_total <= ALBIREO_FIXED_MAX_HISTORY, V <= ALBIREO_MAX_VOCAB; anything
+ * larger returns ALBIREO_EUNSUPPORTED and launches nothing.  Other host-detectable
+ * mistakes return ALBIREO_EINVAL.  The text of the last error on the calling thread is
+ * returned by albireo_sample_fixed_scratch_error().
+ *
+ * First call on each device: looks up the device address of the scratch array and sets
+ * the kernels' shared-memory attributes, with that device current.  Make that first call
+ * before any stream capture on the device; later calls only enqueue a kernel.
+ *
+ * The array is shared by every call in the process and keeps whatever the previous call
+ * left in it.  Nothing has to be cleared by the caller: each row zeroes the counters it is
+ * about to use before counting.  Two calls whose kernels can overlap on the same GPU
+ * (different streams, or threads launching at once) race on the array -- serialise them.
+ */
+int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32_t V, int32_t dtype,
+                                 const float *temperature, const int32_t *top_k,
+                                 const float *top_p, const float *min_p,
+                                 const float *repetition_penalty, const float *presence_penalty,
+                                 const float *frequency_penalty,
+                                 const int32_t *history_ids, const int32_t *history_offsets,
+                                 int64_t history_total,
+                                 const uint64_t *seeds, uint64_t step,
+                                 int32_t *out_tokens, float *out_logprobs,
+                                 void *stream, const albireo_sample_ext_t *ext);
+
+/* Text of the last error albireo_sample_fixed_scratch recorded on the calling thread ("" if none). */
+const char *albireo_sample_fixed_scratch_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,11 +23,12 @@ ROW_GENERAL_PATH, ROW_BAD_PARAM, ROW_HISTORY_OVERFLOW, ROW_TIMEOUT = 1, 2, 4, 8
 FLAG_FORCE_GENERAL = 1
 MAX_VOCAB = 524288
 MAX_NUM_TOP = 128
+FIXED_MAX_HISTORY = 1 << 20
 
 EXPORTS = [
     "albireo_sample_workspace_bytes", "albireo_sample_host_staging_bytes", "albireo_sample_init",
     "albireo_sample", "albireo_sample_host", "albireo_sample_destroy", "albireo_last_error",
-    "albireo_sample_launch_count",
+    "albireo_sample_launch_count", "albireo_sample_fixed_scratch", "albireo_sample_fixed_scratch_error",
 ]
 
 
@@ -69,6 +70,10 @@ def _load() -> C.CDLL:
     lib.albireo_last_error.argtypes = [vp]
     lib.albireo_sample_launch_count.restype = C.c_uint64
     lib.albireo_sample_launch_count.argtypes = [vp]
+    lib.albireo_sample_fixed_scratch.restype = C.c_int
+    lib.albireo_sample_fixed_scratch.argtypes = sample_args[1:14] + [i64] + sample_args[14:]
+    lib.albireo_sample_fixed_scratch_error.restype = C.c_char_p
+    lib.albireo_sample_fixed_scratch_error.argtypes = []
     return lib
 
 
@@ -251,6 +256,44 @@ class Sampler:
         if rc != OK:
             raise AlbireoError(rc, self.last_error())
         return SampleOutputs(out_tokens, out_logprobs, **extra)
+
+
+def albireo_sample_fixed_scratch(logits: torch.Tensor, *, temperature=None, top_k=None, top_p=None, min_p=None,
+                                 repetition_penalty=None, presence_penalty=None, frequency_penalty=None,
+                                 history_ids=None, history_offsets=None, history_total: Optional[int] = None,
+                                 seeds=None, step: int = 0, out_tokens=None, out_logprobs=None,
+                                 stream: Optional[torch.cuda.Stream] = None, row_base: int = 0) -> SampleOutputs:
+    """The sampler for callers that may not allocate: no handle, no workspace (the library's own
+    fixed scratch array is used).  The output tensors created here when none are passed are a
+    convenience of this Python wrapper; the C entry point itself allocates nothing."""
+    B, V = logits.shape
+    dt = F32 if logits.dtype == torch.float32 else BF16
+    if logits.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("logits must be float32 or bfloat16")
+    dev = logits.device
+    if out_tokens is None:
+        out_tokens = torch.empty(B, dtype=torch.int32, device=dev)
+    if out_logprobs is None:
+        out_logprobs = torch.empty(B, dtype=torch.float32, device=dev)
+    ext = SampleExt()
+    ext.struct_size = C.sizeof(SampleExt)
+    ext.row_base = row_base
+    if history_total is None:
+        history_total = int(history_ids.numel()) if history_ids is not None else 0
+    st = torch.cuda.current_stream(dev) if stream is None else stream
+    f32, i32 = torch.float32, torch.int32
+    with torch.cuda.device(dev):
+        rc = LIB.albireo_sample_fixed_scratch(
+            C.c_void_p(logits.data_ptr()), B, V, dt,
+            _dp(temperature, f32, "cuda"), _dp(top_k, i32, "cuda"), _dp(top_p, f32, "cuda"), _dp(min_p, f32, "cuda"),
+            _dp(repetition_penalty, f32, "cuda"), _dp(presence_penalty, f32, "cuda"),
+            _dp(frequency_penalty, f32, "cuda"), _dp(history_ids, i32, "cuda"), _dp(history_offsets, i32, "cuda"),
+            C.c_int64(history_total), _dp(seeds, torch.int64, "cuda"), C.c_uint64(step),
+            C.c_void_p(out_tokens.data_ptr()), C.c_void_p(out_logprobs.data_ptr()),
+            C.c_void_p(st.cuda_stream), C.byref(ext))
+    if rc != OK:
+        raise AlbireoError(rc, LIB.albireo_sample_fixed_scratch_error().decode())
+    return SampleOutputs(out_tokens, out_logprobs)
 
 
 # ------------------------------------------------------------------ workload marshalling

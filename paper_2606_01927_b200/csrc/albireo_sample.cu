@@ -22,6 +22,7 @@
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
+#include <mutex>
 #include <new>
 
 #include "albireo_sample.h"
@@ -1615,3 +1616,129 @@ extern "C" int albireo_sample_destroy(albireo_sampler_t *h) {
 extern "C" const char *albireo_last_error(const albireo_sampler_t *h) { return h ? h->err : ""; }
 
 extern "C" uint64_t albireo_sample_launch_count(const albireo_sampler_t *h) { return h ? h->launches : 0; }
+
+// ------------------------------------------------------------------ entry point that allocates nothing
+//
+// Some callers cannot allocate device memory at the moment they need a sample: a plugin that
+// runs inside a host whose memory pool is already fully handed out, a caller in the middle of
+// work where cudaMalloc would synchronise the device, or code under a rule that forbids
+// allocation after start-up.  For them the history-count scratch that albireo_sample takes from
+// the caller's workspace lives here in a fixed array in the library's own device image.  Every GPU
+// that loads the library holds it (4 MiB) until the process exits.
+
+static __device__ __align__(256) uint32_t g_fixed_counts[ALBIREO_FIXED_MAX_HISTORY];
+
+namespace {
+constexpr int FIXED_MAX_DEVICES = 64;
+struct FixedDeviceState {
+    bool ready;
+    uint32_t *counts;     // device address of g_fixed_counts on that device
+    size_t max_smem;
+};
+FixedDeviceState g_fixed_dev[FIXED_MAX_DEVICES];
+std::mutex g_fixed_mutex;
+thread_local char g_fixed_err[256] = "";
+
+int fixed_fail(int code, const char *fmt, const char *detail) {
+    snprintf(g_fixed_err, sizeof g_fixed_err, fmt, detail ? detail : "");
+    return code;
+}
+
+// Once per device, with that device current: the device address of the scratch array (its name
+// in host code is only a stand-in, never something a kernel may be given) and the kernels'
+// shared-memory opt-in.
+int fixed_setup(int dev, FixedDeviceState **out) {
+    if (dev < 0 || dev >= FIXED_MAX_DEVICES) return fixed_fail(ALBIREO_EUNSUPPORTED, "device index beyond what the fixed-scratch entry supports%s", "");
+    std::lock_guard<std::mutex> lock(g_fixed_mutex);
+    FixedDeviceState &d = g_fixed_dev[dev];
+    if (!d.ready) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_fixed_counts);
+        if (e != cudaSuccess || !ptr) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e)); }
+        int optin = 0;
+        e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        cudaFuncAttributes fa32, fa16;
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa32, albireo_sample_kernel<ALBIREO_F32>);
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa16, albireo_sample_kernel<ALBIREO_BF16>);
+        size_t smem = 0;
+        if (e == cudaSuccess) {
+            const size_t stat = fa32.sharedSizeBytes > fa16.sharedSizeBytes ? fa32.sharedSizeBytes : fa16.sharedSizeBytes;
+            smem = (size_t)optin > stat ? (size_t)optin - stat : 0;
+            e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        }
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "kernel set-up failed: %s", cudaGetErrorString(e)); }
+        d.counts = (uint32_t *)ptr; d.max_smem = smem; d.ready = true;
+    }
+    *out = &d;
+    return ALBIREO_OK;
+}
+}  // namespace
+
+extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32_t V, int32_t dtype,
+                                            const float *temperature, const int32_t *top_k, const float *top_p,
+                                            const float *min_p, const float *repetition_penalty,
+                                            const float *presence_penalty, const float *frequency_penalty,
+                                            const int32_t *history_ids, const int32_t *history_offsets,
+                                            int64_t history_total, const uint64_t *seeds, uint64_t step,
+                                            int32_t *out_tokens, float *out_logprobs, void *stream,
+                                            const albireo_sample_ext_t *ext) {
+    g_fixed_err[0] = 0;
+    if (B == 0) return ALBIREO_OK;
+    if (B < 0) return fixed_fail(ALBIREO_EINVAL, "B is negative%s", "");
+    if (V < 1) return fixed_fail(ALBIREO_EINVAL, "V is not positive%s", "");
+    if (V > ALBIREO_MAX_VOCAB) return fixed_fail(ALBIREO_EUNSUPPORTED, "V exceeds ALBIREO_MAX_VOCAB%s", "");
+    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16) return fixed_fail(ALBIREO_EINVAL, "unknown dtype%s", "");
+    if (!logits || !out_tokens || !out_logprobs) return fixed_fail(ALBIREO_EINVAL, "NULL logits or output%s", "");
+    if ((history_ids == nullptr) != (history_offsets == nullptr)) return fixed_fail(ALBIREO_EINVAL, "history_ids and history_offsets must both be given%s", "");
+    if (history_total < 0) return fixed_fail(ALBIREO_EINVAL, "history_total is negative%s", "");
+    if (history_total > (int64_t)ALBIREO_FIXED_MAX_HISTORY)
+        return fixed_fail(ALBIREO_EUNSUPPORTED, "history_total exceeds ALBIREO_FIXED_MAX_HISTORY (the fixed scratch array); use albireo_sample with a workspace%s", "");
+    const size_t esize = dtype == ALBIREO_F32 ? 4 : 2;
+    if ((uintptr_t)logits % esize) return fixed_fail(ALBIREO_EINVAL, "logits not element-aligned%s", "");
+
+    SampleArgs a;
+    memset(&a, 0, sizeof a);
+    a.logits = logits; a.B = B; a.V = V; a.row_stride = V;
+    a.temperature = temperature; a.top_k = top_k; a.top_p = top_p; a.min_p = min_p;
+    a.rep = repetition_penalty; a.pres = presence_penalty; a.freq = frequency_penalty;
+    a.hist_ids = history_ids; a.hist_off = history_offsets;
+    a.seeds = seeds; a.step = step;
+    a.out_tokens = out_tokens; a.out_logprobs = out_logprobs;
+    if (ext) {
+        if (ext->struct_size != sizeof(albireo_sample_ext_t)) return fixed_fail(ALBIREO_EINVAL, "ext->struct_size mismatch%s", "");
+        if (ext->row_stride_elems != 0) {
+            if (ext->row_stride_elems < V) return fixed_fail(ALBIREO_EINVAL, "row stride smaller than V%s", "");
+            a.row_stride = ext->row_stride_elems;
+        }
+        a.row_base = ext->row_base; a.flags = ext->flags;
+        if (ext->num_top < 0 || ext->num_top > ALBIREO_MAX_NUM_TOP) return fixed_fail(ALBIREO_EUNSUPPORTED, "num_top out of range%s", "");
+        if (ext->num_top > 0 && (!ext->out_top_ids || !ext->out_top_logprobs)) return fixed_fail(ALBIREO_EINVAL, "num_top > 0 needs both top-N outputs%s", "");
+        a.num_top = ext->num_top; a.out_top_ids = ext->out_top_ids; a.out_top_logprobs = ext->out_top_logprobs;
+        a.out_num_kept = ext->out_num_kept; a.out_num_topk = ext->out_num_topk;
+        if (ext->dbg_cap < 0 || (ext->dbg_cap > 0 && !ext->dbg_topk_ids)) return fixed_fail(ALBIREO_EINVAL, "bad dbg_cap / dbg_topk_ids%s", "");
+        a.dbg_cap = ext->dbg_topk_ids ? ext->dbg_cap : 0;
+        a.dbg_topk_ids = ext->dbg_cap > 0 ? ext->dbg_topk_ids : nullptr;
+        a.out_row_status = ext->out_row_status;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "cudaGetDevice failed%s", ""); }
+    FixedDeviceState *d = nullptr;
+    const int rc = fixed_setup(dev, &d);
+    if (rc != ALBIREO_OK) return rc;
+    a.ws_counts = d->counts;                       // a device address, from cudaGetSymbolAddress
+    a.ws_counts_cap = ALBIREO_FIXED_MAX_HISTORY;
+
+    a.nstages = ring_stages_for(V, history_ids != nullptr);
+    size_t smem = smem_bytes_for(V, history_ids != nullptr, a.nstages);
+    while (smem > d->max_smem && a.nstages > 2) smem = smem_bytes_for(V, history_ids != nullptr, --a.nstages);
+    if (smem > d->max_smem) return fixed_fail(ALBIREO_EUNSUPPORTED, "vocabulary too large for the on-chip tables%s", "");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == ALBIREO_F32) albireo_sample_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(a);
+    else albireo_sample_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(a);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fixed_fail(ALBIREO_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    return ALBIREO_OK;
+}
+
+extern "C" const char *albireo_sample_fixed_scratch_error(void) { return g_fixed_err; }
