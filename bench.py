@@ -320,13 +320,20 @@ def main():
             "clocks": clock_info,
         }
         if world == 1 and not args.skip_cpu_baseline:
+            # the oracle as it stands on the machine's cores: whole batches until ~15 s of CPU work are done
             from oracle import albireo_oracle as O
             cores = len(os.sched_getaffinity(0))
-            t0 = time.perf_counter()
-            O.sample(w, threads=cores)
-            dt = time.perf_counter() - t0
-            line["cpu_baseline"] = {"value": w.B / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": f"all {w.B} rows of the batch once, one thread per core ({dt:.2f} s wall)"}
+            reps, cpu_s, best = 0, 0.0, float("inf")
+            while reps < 2 or (cpu_s < 15.0 and reps < 32):
+                t0 = time.perf_counter()
+                O.sample(w, threads=cores)
+                dt = time.perf_counter() - t0
+                best = min(best, dt)
+                cpu_s += dt * cores
+                reps += 1
+            line["cpu_baseline"] = {"value": w.B / best, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"all {w.B} rows of the batch, {reps} passes (best of them), one thread per core, "
+                                              f"~{cpu_s:.0f} s of CPU work in total"}
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
