@@ -36,8 +36,9 @@ N_ROTATING = 8            # distinct logits buffers, so that no call finds its r
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of albireo_sample_kernel on the
-# metric workload, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"configM": None}
+# metric workload, from the ncu capture summarised in profiles/albireo_sample_kernel_configM.md
+# (mean of the two captured launches).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"configM": 79680384}
 
 
 def measured_peak():
@@ -162,6 +163,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch each step from Python instead of one CUDA graph")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--general-path", action="store_true", help="force every row down the general path")
+    ap.add_argument("--read-ceiling", action="store_true",
+                    help="only run the read-ceiling tool (a kernel that just reads the same bytes) and print its table")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -174,6 +177,12 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             run_reference(args, W.make(args.workload))
+        return
+    if args.read_ceiling:
+        if rank == 0:
+            import subprocess
+            from paper_2606_01927_b200 import _build as B_
+            print(subprocess.run([B_.build_tools()], capture_output=True, text=True).stdout)
         return
 
     import torch
