@@ -910,25 +910,39 @@ __device__ __forceinline__ void cand_append_one(BlockScratch &s, const CandSmem 
 __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, float zmax, bool has_minp,
                             const RowParams &rp, const SampleArgs &a, int b, RowOut &out) {
     const int lane = threadIdx.x & 31;
+    // `parts` threads share one candidate's comparisons; the threads after them (from the next warp
+    // boundary on) take one candidate each for the race term and the mass, so those long dependent
+    // chains run with full lanes and beside the rank loops instead of after them.
     int parts = 1;
-    while (parts < 8 && n * parts * 2 <= NT) parts *= 2;
+    while (parts < 8 && ((n * parts * 2 + 31) & ~31) + n <= NT) parts *= 2;
+    const int dstart = (n * parts + 31) & ~31;
+    const bool dense_ok = dstart + n <= NT;
     const int j = threadIdx.x / parts, part = threadIdx.x % parts;
+    float *nle = (float *)(cs.gsc + SORT_MAX);           // n race terms, then n masses (as u64) behind them
+    u64 *mass = (u64 *)(nle + SORT_MAX);
     u64 C = 0;
     int rank = 0;
-    float g = 0.0f;
     if (j < n) {
         C = cs.cand[j];
-        if (part == 0) g = neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, comp_idx(C)));
         for (int q = part; q < n; q += parts) rank += cs.cand[q] > C;
     }
+    {
+        const int t = dense_ok ? (int)threadIdx.x - dstart : (part == 0 ? j : -1);
+        if (t >= 0 && t < n) {
+            const u64 Ct = cs.cand[t];
+            nle[t] = neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, comp_idx(Ct)));
+            mass[t] = mass_fx(__fsub_rn(unkey((uint32_t)(Ct >> 32)), zmax));
+        }
+    }
     for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+    __syncthreads();
     bool in7 = false;
     if (j < n && part == 0) {
         const float z = unkey((uint32_t)(C >> 32));
         const float d = __fsub_rn(z, zmax);
         cs.sorted[rank] = C;
-        cs.efx[rank] = mass_fx(d);
-        cs.gsc[rank] = ((u64)orderable_f32(d + g) << 32) | (uint32_t)C;
+        cs.efx[rank] = mass[j];
+        cs.gsc[rank] = ((u64)orderable_f32(d + nle[j]) << 32) | (uint32_t)C;
         in7 = rank < L6 && (!has_minp || ((double)z - (double)zmax >= log((double)rp.min_p)));
     }
     // min-p keeps a prefix of the order, at least one element (the barrier also publishes step 1)
