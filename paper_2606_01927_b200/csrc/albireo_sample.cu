@@ -952,34 +952,33 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         a.dbg_topk_ids[(int64_t)b * a.dbg_cap + threadIdx.x] = comp_idx(cs.sorted[threadIdx.x]);
     if (threadIdx.x >= 32) return;
 
-    const u64 *sorted = cs.sorted, *gsc = cs.gsc;
-    u64 *efx = cs.efx;
-    // Masses are fixed point: integer sums are exact, so the prefix sums do not depend on the
-    // order of the additions.  Inclusive prefix sums replace the masses in place.
-    u64 carry = 0;
-    for (int q0 = 0; q0 < L7; q0 += 32) {
-        const int q = q0 + lane;
-        u64 inc = q < L7 ? efx[q] : 0ull;
+    const u64 *sorted = cs.sorted, *gsc = cs.gsc, *efx = cs.efx;
+    // Each lane owns a contiguous run of the sorted list.  Masses are fixed point: integer sums are
+    // exact, so the prefix sums do not depend on the order of the additions.
+    const int per = (L7 + 31) >> 5;
+    const int q0 = lane * per, q1 = min(L7, q0 + per);
+    u64 local = 0;
+    for (int q = q0; q < q1; ++q) local += efx[q];
+    u64 incl = local;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t2; }
-        inc += carry;
-        if (q < L7) efx[q] = inc;
-        carry = __shfl_sync(0xFFFFFFFFu, inc, 31);
-    }
-    const u64 tot = carry;
+    for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t2; }
+    const u64 tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
     int L8 = L7;
     u64 S_fx = tot;
     if (!rp.greedy && rp.top_p < 1.0f) {
         double t = ceil((double)rp.top_p * (double)tot);
         u64 target = t <= 1.0 ? 1ull : (u64)t;
         if (target > tot) target = tot;
-        __syncwarp();
-        // smallest prefix whose mass reaches the target: count the elements whose inclusive sum is below it
-        int below = 0;
-        for (int q = lane; q < L7; q += 32) below += efx[q] < target;
-        below = __reduce_add_sync(0xFFFFFFFFu, below);
-        L8 = below + 1 < L7 ? below + 1 : L7;
-        S_fx = efx[L8 - 1];
+        // smallest prefix whose mass reaches the target: keep an element while the mass ahead of it is short
+        u64 run = incl - local, last = 0;
+        int cnt = 0;
+        for (int q = q0; q < q1; ++q) {
+            const bool keep = run < target;
+            run += efx[q];
+            if (keep) { ++cnt; last = run; }
+        }
+        L8 = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        S_fx = __shfl_sync(0xFFFFFFFFu, last, (L8 - 1) / per);
     }
     const float lnS = logf((float)S_fx * (1.0f / FX_SCALE));
     int tok = comp_idx(sorted[0]);
@@ -987,7 +986,7 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
     if (L8 > 1) {
         // argmax of the race score over the kept prefix (ties: lowest id, via the low word ~id)
         u64 best = 0; int bestq = 0;
-        for (int q = lane; q < L8; q += 32) { u64 G = gsc[q]; if (G > best) { best = G; bestq = q; } }
+        for (int q = q0; q < min(q1, L8); ++q) { u64 G = gsc[q]; if (G > best) { best = G; bestq = q; } }
         const uint32_t ghi = __reduce_max_sync(0xFFFFFFFFu, (uint32_t)(best >> 32));
         const uint32_t glo = __reduce_max_sync(0xFFFFFFFFu, (uint32_t)(best >> 32) == ghi ? (uint32_t)best : 0u);
         const uint32_t who = __ballot_sync(0xFFFFFFFFu, (uint32_t)(best >> 32) == ghi && (uint32_t)best == glo);
