@@ -1050,7 +1050,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     cs.hist[threadIdx.x] = 0;
     __syncthreads();
 
-    uint32_t tau_key = KEY_MIN_FINITE;
+    uint32_t tau_topk = KEY_MIN_FINITE;   // the top-k part of the threshold: identical in every thread
+    uint32_t tau_key = KEY_MIN_FINITE;    // the threshold in use: max(tau_topk, min-p floor this warp has seen)
     uint32_t thr = 0;
     uint32_t seen_max = 0;
     const uint32_t trig0 = has_topk ? (uint32_t)min(CAND_CAP / 2, 4 * k + 64) : (uint32_t)(CAND_CAP / 2);
@@ -1060,15 +1061,23 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         // warm-up on the first NT vectors: the k-th largest of the per-thread maxima (each an
         // unpenalised element of the row, all distinct) is a lower bound of the row's k-th
         // largest score
+        // (a large k needs a larger sample to give a useful bound: then the whole first tile)
+        const int wvecs = (has_topk && k > 64) ? TILE_VECS : 1;
         bool bad = !mbar_wait(&rg.bar[MAX_STAGES - 1], 0);
+        if (wvecs > 1 && !bad) bad = !mbar_wait(&rg.bar[0], 0);
         uint32_t mk = 0;
-        if (pvec < nvec && !bad) {
-            const uint4 q = ((const uint4 *)rg.buf)[pvec];
-            const int i0 = head + pvec * E::PER_VEC;
-            if (c.has_hist && (__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u)))
-                mk = masked_vmax_key<DT>(c, q, i0);
-            else
-                mk = T::vmax_key(q, c.invT);
+        for (int u = 0; u < wvecs; ++u) {
+            const int v = u * NT + pvec;
+            if (v < nvec && !bad) {
+                const uint4 q = ((const uint4 *)rg.buf)[v];
+                const int i0 = head + v * E::PER_VEC;
+                uint32_t kk;
+                if (c.has_hist && (__funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u)))
+                    kk = masked_vmax_key<DT>(c, q, i0);
+                else
+                    kk = T::vmax_key(q, c.invT);
+                mk = kk > mk ? kk : mk;
+            }
         }
         if (mk < KEY_MIN_FINITE || mk >= KEY_POS_INF) mk = 0;
         cs.cand[threadIdx.x] = (u64)mk << 32;
@@ -1084,8 +1093,9 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         // fewer than k valid maxima: the select fails and tau stays at its floor
         if (has_topk && kmax) {
             uint32_t kk = (uint32_t)k, lo = kmin, hi = kmax; int shift;
-            if (cand_select_pass(s, cs, NT, kk, lo, hi, shift, true)) tau_key = lo;
+            if (cand_select_pass(s, cs, NT, kk, lo, hi, shift, true)) tau_topk = lo;
         }
+        tau_key = tau_topk;
         if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
         seen_max = kmax;
         thr = T::raw_threshold(tau_key, c.invT);
@@ -1101,39 +1111,47 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     int st = 0;                      // ring stage of the current tile
     uint32_t parity = 0;             // its mbarrier phase
     for (int tile = 0; tile < ntiles; ++tile) {
-        if ((uint32_t)tile == *(volatile uint32_t *)&s.maint_at) {
+        // Tile 0 holds the head of the vocabulary and is the densest; right after it the list is
+        // looked at once in any case (a bound from 4x the warm-up sample is much tighter).
+        if ((uint32_t)tile == *(volatile uint32_t *)&s.maint_at || tile == 1) {
             __syncthreads();                       // every warp is between tiles: nobody appends
             int n = (int)s.cand_cnt;
             const uint32_t ovf = s.overflow, rmax = s.runmax, tmo = s.timeout;
             __syncthreads();
-            if (threadIdx.x == 0) s.maint_at = 0xFFFFFFFFu;
+            if (threadIdx.x == 0 && (uint32_t)tile == s.maint_at) s.maint_at = 0xFFFFFFFFu;
             if (ovf || tmo) {
                 ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
                 if (tmo) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; return true; }
                 __syncthreads();
                 return false;
             }
-            bool changed = false;
-            if (stream_minp && rmax > seen_max) {
-                seen_max = rmax;
-                uint32_t f = minp_key(unkey(rmax), rp.min_p);
-                if (f > tau_key) { tau_key = f; changed = true; }
-            }
-            if ((uint32_t)n + 1u >= trig) {
+            // make the threshold identical in every thread again
+            uint32_t tau_new = tau_topk;
+            if (stream_minp && rmax) { seen_max = rmax; uint32_t f = minp_key(unkey(rmax), rp.min_p); tau_new = f > tau_new ? f : tau_new; }
+            const uint32_t trig_now = (tile == 1) ? min(trig, (uint32_t)(has_topk ? 2 * k + 32 : CAND_CAP / 4)) : trig;
+            if ((uint32_t)n + 1u >= trig_now) {
                 if (has_topk && n >= k) {
-                    uint32_t lmx = 0, mn, hi;
-                    for (int i = threadIdx.x; i < n; i += NT) { uint32_t kk = (uint32_t)(cs.cand[i] >> 32); lmx = kk > lmx ? kk : lmx; }
-                    block_minmax_u32(s, lmx, mn, hi);
-                    uint32_t t = cand_select_approx(s, cs, n, k, tau_key, hi);
-                    if (t > tau_key) { tau_key = t; changed = true; }
+                    uint32_t t = cand_select_approx(s, cs, n, k, tau_topk, rmax);
+                    if (t > tau_topk) tau_topk = t;
+                    if (t > tau_new) tau_new = t;
                 }
-                n = cand_compact(s, cs, n, tau_key);
+                n = cand_compact(s, cs, n, tau_new);
                 // if the list could not be shrunk (ties), look again only after it has grown
                 trig = (uint32_t)n + (uint32_t)(has_topk ? 2 * k + 32 : CAND_CAP / 4);
                 if (trig < trig0) trig = trig0;
             }
-            if (changed) thr = T::raw_threshold(tau_key, c.invT);
+            if (tau_new != tau_key) { tau_key = tau_new; thr = T::raw_threshold(tau_key, c.invT); }
             __syncthreads();                       // s.maint_at is reset before anyone asks again
+        }
+        if (stream_minp) {
+            // the min-p floor follows the running maximum without any block-wide step: a warp that
+            // still uses an older (lower) floor is merely less selective
+            const uint32_t rm = *(volatile uint32_t *)&s.runmax;
+            if (rm > seen_max) {
+                seen_max = rm;
+                const uint32_t f = minp_key(unkey(rm), rp.min_p);
+                if (f > tau_key) { tau_key = f; thr = T::raw_threshold(tau_key, c.invT); }
+            }
         }
         const int vbase = tile * NT * TILE_VECS;
         bool ask = false;                          // ask for a rendezvous
@@ -1190,7 +1208,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
                             lmax = __reduce_max_sync(0xFFFFFFFFu, lmax);
                             if (lane == 0 && lmax > *(volatile uint32_t *)&s.runmax) {
                                 const uint32_t old = atomicMax(&s.runmax, lmax);
-                                ask = ask || (stream_minp && lmax > old && lmax > seen_max);
+                                (void)old;
                             }
 
                         }
