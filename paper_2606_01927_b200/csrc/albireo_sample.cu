@@ -332,124 +332,29 @@ __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, co
     return true;
 }
 
-// ------------------------------------------------------------------ general path: radix selection
+// ------------------------------------------------------------------ general path: histogram selection
+//
+// For rows the candidate path does not take (top-p without top-k, no cuts at all, a top-k above
+// 256, or a candidate list that would overflow).  The kept set is a prefix of the total order, i.e.
+// { t : C(t) >= C_cut }; the cut is found exactly with a few passes over the row (re-read from L2):
+//   pass 0  the largest composite (z_max and its id) and the number of finite scores;
+//   pass 1  a 2048-bin histogram (count, and 2^40 fixed-point mass) over value-linear bins of
+//           z_max - z (1/32 wide), so that elements spread over many bins;
+//   cut     the bin in which the wanted rank or mass falls; its elements are gathered into shared
+//           memory and the exact position is found there (a bin too full for that is first narrowed
+//           with composite-linear histograms over the row);
+//   final   the race over the kept set, its mass and its size.
 
 struct HistBins {
     uint32_t *cnt;   // HIST_BINS
     u64 *mass;       // HIST_BINS
+    u64 *list;       // GL_CAP composites gathered from the row
+    u64 *acc;        // SEL_ACC bins for the on-chip search in the list
 };
 
-__constant__ int LVL_SHIFT[6] = {53, 42, 32, 21, 10, 0};
-__constant__ int LVL_BITS[6] = {11, 11, 10, 11, 11, 10};
-
-// Scans bins from the highest digit down and finds the bin where the running total first
-// reaches `target` (target >= 1, <= grand total).  use_mass selects which histogram steers.
-// Returns digit, the total strictly above the bin, and the bin's element count.
-__device__ void find_bin(BlockScratch &s, const HistBins &h, int nbins, bool use_mass, u64 target,
-                         uint32_t &digit, u64 &above, uint32_t &bin_cnt) {
-    // thread t owns bins [nbins - per*(t+1), nbins - per*t), visited from the top
-    const int per = (nbins + NT - 1) / NT;
-    u64 local = 0;
-    for (int q = 0; q < per; ++q) {
-        int bin = nbins - 1 - (threadIdx.x * per + q);
-        if (bin >= 0) local += use_mass ? h.mass[bin] : (u64)h.cnt[bin];
-    }
-    u64 tot;
-    u64 run = block_exscan_u64(s, local, tot);
-    if (threadIdx.x == 0) { s.found_digit = 0xFFFFFFFFu; s.found_cnt = 0; s.found_above = 0; }
-    __syncthreads();
-    if (run < target && target <= run + local) {
-        for (int q = 0; q < per; ++q) {
-            int bin = nbins - 1 - (threadIdx.x * per + q);
-            if (bin < 0) break;
-            u64 v = use_mass ? h.mass[bin] : (u64)h.cnt[bin];
-            if (run < target && target <= run + v) {
-                s.found_digit = (uint32_t)bin; s.found_above = run; s.found_cnt = h.cnt[bin];
-                break;
-            }
-            run += v;
-        }
-    }
-    __syncthreads();
-    digit = s.found_digit; above = s.found_above; bin_cnt = s.found_cnt;
-}
-
-// Selection by count: returns the composite of the `rank`-th largest element (1-based)
-// among { C >= lo } whose top bits (above level `lvl0`) equal `prefix`.
-// Precondition: 1 <= rank <= number of such elements.
-template <int DT>
-__device__ u64 select_by_count(BlockScratch &s, const HistBins &h, const RowCtx &c, u64 lo, u64 rank,
-                               int lvl0, u64 prefix) {
-    for (int lvl = lvl0; lvl < 6; ++lvl) {
-        const int shift = LVL_SHIFT[lvl], bits = LVL_BITS[lvl], nbins = 1 << bits;
-        if (lvl == 3 && c.V <= (1 << 21)) { prefix = (prefix << 11) | 0x7FFu; continue; }  // ~id has these bits all set
-        for (int bnum = threadIdx.x; bnum < nbins; bnum += NT) h.cnt[bnum] = 0;
-        __syncthreads();
-        const int up = shift + bits;
-        for_each_score<DT>(c, [&](int i, float z) {
-            u64 C = comp_of(key_of(z), i);
-            bool in = C >= lo && (up >= 64 || (C >> up) == prefix);
-            if (in) atomicAdd(&h.cnt[(uint32_t)(C >> shift) & (nbins - 1)], 1u);
-        });
-        __syncthreads();
-        uint32_t digit, bin_cnt; u64 above;
-        find_bin(s, h, nbins, false, rank, digit, above, bin_cnt);
-        if (digit == 0xFFFFFFFFu) return lo;            // precondition violated; keep everything
-        rank -= above;
-        prefix = (prefix << bits) | digit;
-        if (rank == bin_cnt) {                           // the whole bin is taken
-            u64 t = prefix << shift;
-            return t > lo ? t : lo;
-        }
-    }
-    return prefix;
-}
-
-// Selection by mass: smallest prefix of { C >= lo } whose mass reaches top_p times the
-// mass of the whole set.  Returns its composite threshold.
-template <int DT>
-__device__ u64 select_by_mass(BlockScratch &s, const HistBins &h, const RowCtx &c, u64 lo, float zmax, float top_p) {
-    u64 prefix = 0, target = 0;
-    uint32_t bin_cnt = 0;
-    for (int lvl = 0; lvl < 3; ++lvl) {
-        const int shift = LVL_SHIFT[lvl], bits = LVL_BITS[lvl], nbins = 1 << bits;
-        for (int bnum = threadIdx.x; bnum < nbins; bnum += NT) { h.cnt[bnum] = 0; h.mass[bnum] = 0; }
-        __syncthreads();
-        const int up = shift + bits;
-        for_each_score<DT>(c, [&](int i, float z) {
-            u64 C = comp_of(key_of(z), i);
-            bool in = C >= lo && (up >= 64 || (C >> up) == prefix);
-            if (in) {
-                uint32_t d = (uint32_t)(C >> shift) & (nbins - 1);
-                atomicAdd(&h.cnt[d], 1u);
-                atomicAdd(&h.mass[d], mass_fx(__fsub_rn(z, zmax)));
-            }
-        });
-        __syncthreads();
-        if (lvl == 0) {
-            u64 local = 0;
-            for (int bnum = threadIdx.x; bnum < nbins; bnum += NT) local += h.mass[bnum];
-            u64 total = block_sum_u64(s, local);
-            double t = ceil((double)top_p * (double)total);
-            target = t <= 1.0 ? 1ull : (u64)t;
-            if (target > total) target = total;
-            if (target < 1) target = 1;
-        }
-        uint32_t digit; u64 above;
-        find_bin(s, h, nbins, true, target, digit, above, bin_cnt);
-        if (digit == 0xFFFFFFFFu) return lo;
-        target -= above;
-        prefix = (prefix << bits) | digit;
-    }
-    // prefix is now a full key; bin_cnt ties share one mass value each
-    const uint32_t tkey = (uint32_t)prefix;
-    u64 e1 = mass_fx(__fsub_rn(unkey(tkey), zmax));
-    u64 m = e1 ? (target + e1 - 1) / e1 : bin_cnt;
-    if (m < 1) m = 1;
-    u64 tie_lo = ((u64)tkey << 32) > lo ? ((u64)tkey << 32) : lo;
-    if (m >= bin_cnt) return tie_lo;
-    return select_by_count<DT>(s, h, c, tie_lo, m, 3, (u64)tkey);
-}
+constexpr int GL_CAP = 2048;
+constexpr int SEL_ACC = NT;             // one accumulator per thread
+constexpr float BIN_SCALE = 32.0f;      // bins per unit of z
 
 struct RowParams {
     float T, top_p, min_p;
@@ -480,25 +385,142 @@ __device__ uint32_t minp_key(float zmax, float min_p) {
     return k < KEY_MIN_FINITE ? KEY_MIN_FINITE : k;
 }
 
-// Gathers { C >= thr } (at most cap of them) into list[], sorted best first.  list must
-// hold cap entries.  Returns the number gathered (elements beyond cap are dropped).
-template <int DT>
-__device__ int gather_sorted(BlockScratch &s, const RowCtx &c, u64 thr, u64 *list, u64 *tmp, int cap) {
-    if (threadIdx.x == 0) s.list_cnt = 0;
+// value-linear bin of a finite score z <= zmax; monotone: a larger z never gets a larger bin
+__device__ __forceinline__ int bin_of(float z, float zmax) {
+    int b = __float2int_rz(__fsub_rn(zmax, z) * BIN_SCALE);
+    return b < 0 ? 0 : (b > HIST_BINS - 1 ? HIST_BINS - 1 : b);
+}
+__device__ __forceinline__ int bitlen64(u64 v) { return 64 - __clzll((long long)v); }
+
+// Finds the first bin (from bin 0) at which the running total of the steering histogram reaches
+// `target` (1 <= target <= grand total).  Gives the totals of both histograms strictly before it.
+__device__ bool find_prefix_bin(BlockScratch &s, const HistBins &h, bool by_mass, bool have_mass, u64 target,
+                                int &bin, u64 &cnt_before, u64 &mass_before) {
+    constexpr int PER = HIST_BINS / NT;
+    u64 lc = 0, lm = 0;
+#pragma unroll
+    for (int q = 0; q < PER; ++q) { lc += h.cnt[threadIdx.x * PER + q]; if (have_mass) lm += h.mass[threadIdx.x * PER + q]; }
+    u64 totc, totm = 0;
+    u64 runc = block_exscan_u64(s, lc, totc);
+    u64 runm = have_mass ? block_exscan_u64(s, lm, totm) : 0ull;
+    if (threadIdx.x == 0) s.found_digit = 0xFFFFFFFFu;
     __syncthreads();
-    for_each_score<DT>(c, [&](int i, float z) {
-        u64 C = comp_of(key_of(z), i);
-        if (C >= thr) { uint32_t slot = atomicAdd(&s.list_cnt, 1u); if (slot < (uint32_t)cap) tmp[slot] = C; }
-    });
-    __syncthreads();
-    int n = min((int)s.list_cnt, cap);
-    for (int a = threadIdx.x; a < n; a += NT) {
-        u64 C = tmp[a]; int rank = 0;
-        for (int b2 = 0; b2 < n; ++b2) rank += tmp[b2] > C;
-        list[rank] = C;
+    const u64 run = by_mass ? runm : runc, loc = by_mass ? lm : lc;
+    if (run < target && target <= run + loc) {
+        u64 rc = runc, rm = runm;
+        for (int q = 0; q < PER; ++q) {
+            const int bq = threadIdx.x * PER + q;
+            const u64 vc = h.cnt[bq], vm = have_mass ? h.mass[bq] : 0ull;
+            const u64 r = by_mass ? rm : rc, v = by_mass ? vm : vc;
+            if (r < target && target <= r + v) { s.found_digit = (uint32_t)bq; s.found_above = rc; s.bcast[2] = rm; break; }
+            rc += vc; rm += vm;
+        }
     }
     __syncthreads();
-    return n;
+    if (s.found_digit == 0xFFFFFFFFu) return false;
+    bin = (int)s.found_digit; cnt_before = s.found_above; mass_before = s.bcast[2];
+    return true;
+}
+
+// Gathers the composites accepted by `take` into h.list (at most GL_CAP are stored); returns how many
+// were accepted, and their smallest and largest composite.
+template <int DT, class F>
+__device__ int gather_if(BlockScratch &s, const HistBins &h, const RowCtx &c, F &&take, u64 &cmin, u64 &cmax) {
+    if (threadIdx.x == 0) s.list_cnt = 0;
+    __syncthreads();
+    u64 mn = ~0ull, mx = 0;
+    for_each_score<DT>(c, [&](int i, float z) {
+        const u64 C = comp_of(key_of(z), i);
+        if (take(C, z)) {
+            const uint32_t slot = atomicAdd(&s.list_cnt, 1u);
+            if (slot < (uint32_t)GL_CAP) h.list[slot] = C;
+            mn = C < mn ? C : mn; mx = C > mx ? C : mx;
+        }
+    });
+    cmax = block_max_u64(s, mx);
+    cmin = ~block_max_u64(s, ~mn);
+    return (int)s.list_cnt;
+}
+
+// On-chip: in h.list[0..n) (distinct composites within [lo, hi]) find the composite at which the
+// running total, taken from the largest composite down, first reaches `target` -- counting
+// elements (by_mass = false) or their masses.  Range-adaptive bins, repeated until a bin is one value.
+__device__ u64 list_resolve(BlockScratch &s, const HistBins &h, int n, bool by_mass, u64 target, u64 lo, u64 hi, float zmax) {
+    for (int pass = 0; pass < 8; ++pass) {
+        const u64 width = hi - lo;
+        const int shift = width < (u64)SEL_ACC ? 0 : bitlen64(width) - 9;
+        h.acc[threadIdx.x] = 0;
+        if (threadIdx.x == 0) s.found_digit = 0xFFFFFFFFu;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += NT) {
+            const u64 C = h.list[i];
+            if (C >= lo && C <= hi) {
+                const u64 v = by_mass ? mass_fx(__fsub_rn(unkey((uint32_t)(C >> 32)), zmax)) : 1ull;
+                atomicAdd(&h.acc[(hi - C) >> shift], v);
+            }
+        }
+        __syncthreads();
+        const u64 mine = h.acc[threadIdx.x];
+        u64 tot;
+        const u64 before = block_exscan_u64(s, mine, tot);
+        if (before < target && target <= before + mine) { s.found_digit = threadIdx.x; s.found_above = before; }
+        __syncthreads();
+        if (s.found_digit == 0xFFFFFFFFu) return lo;          // target beyond the list: keep all of it
+        const u64 b = s.found_digit;
+        target -= s.found_above;
+        const u64 nhi = hi - (b << shift);
+        if (shift == 0) return nhi;
+        const u64 span = (1ull << shift) - 1ull;
+        lo = (nhi - lo > span) ? nhi - span : lo;
+        hi = nhi;
+        __syncthreads();
+    }
+    return lo;
+}
+
+// Exact cut inside the row: the composite at which the running total (count or mass, from the top of
+// the order, over elements with C >= floorC) first reaches `target`, given that it falls in value bin
+// `bin` and that `before` of the total lies in the bins ahead of it.
+template <int DT>
+__device__ u64 resolve_cut(BlockScratch &s, const HistBins &h, const RowCtx &c, float zmax, int bin, bool by_mass,
+                           u64 target, u64 before, u64 floorC) {
+    u64 rel = target - before;
+    u64 lo, hi;
+    int n = gather_if<DT>(s, h, c, [&](u64 C, float z) { return C >= floorC && (C >> 32) < KEY_POS_INF && bin_of(z, zmax) == bin; }, lo, hi);
+    // a bin too full for the list is narrowed with composite-linear histograms over the row
+    for (int it = 0; it < 8 && n > GL_CAP; ++it) {
+        const u64 width = hi - lo;
+        const int shift = width < (u64)HIST_BINS ? 0 : bitlen64(width) - 11;
+        for (int q = threadIdx.x; q < HIST_BINS; q += NT) { h.cnt[q] = 0; h.mass[q] = 0; }
+        __syncthreads();
+        for_each_score<DT>(c, [&](int i, float z) {
+            const u64 C = comp_of(key_of(z), i);
+            if (C >= lo && C <= hi && C >= floorC) {
+                const uint32_t q = (uint32_t)((hi - C) >> shift);
+                atomicAdd(&h.cnt[q], 1u);
+                if (by_mass) atomicAdd(&h.mass[q], mass_fx(__fsub_rn(z, zmax)));
+            }
+        });
+        __syncthreads();
+        int sub; u64 cb, mb;
+        if (!find_prefix_bin(s, h, by_mass, by_mass, rel, sub, cb, mb)) return lo > floorC ? lo : floorC;
+        rel -= by_mass ? mb : cb;
+        const u64 nhi = hi - ((u64)sub << shift);
+        if (shift == 0) return nhi;
+        const u64 span = (1ull << shift) - 1ull;
+        const u64 nlo = (nhi - lo > span) ? nhi - span : lo;
+        n = (int)h.cnt[sub];
+        __syncthreads();
+        lo = nlo; hi = nhi;
+        if (n <= GL_CAP) {
+            u64 l2, h2;
+            n = gather_if<DT>(s, h, c, [&](u64 C, float) { return C >= lo && C <= hi && C >= floorC; }, l2, h2);
+            lo = l2; hi = h2;
+        }
+    }
+    if (n > GL_CAP) return lo > floorC ? lo : floorC;        // not reachable: composites are distinct
+    if (n < 1) return floorC;
+    return list_resolve(s, h, n, by_mass, rel, lo, hi, zmax);
 }
 
 template <int DT>
@@ -528,13 +550,37 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         return;
     }
 
-    // top-k stage
     const u64 Cfin = (u64)KEY_MIN_FINITE << 32;
+    const bool want_k = rp.top_k >= 1 && rp.top_k < V && (u64)rp.top_k < n_fin;
+    const bool want_minp = rp.min_p > 0.0f;
+    const bool want_topp = rp.top_p < 1.0f;
+    const bool want_top_list = a.num_top > 0;
+    bool have_hist = false;
+    auto build_hist = [&](bool with_mass) {
+        for (int q = threadIdx.x; q < HIST_BINS; q += NT) { h.cnt[q] = 0; h.mass[q] = 0; }
+        __syncthreads();
+        for_each_score<DT>(c, [&](int, float z) {
+            const uint32_t k = key_of(z);
+            if (k >= KEY_MIN_FINITE && k < KEY_POS_INF) {
+                const int q = bin_of(z, zmax);
+                atomicAdd(&h.cnt[q], 1u);
+                if (with_mass) atomicAdd(&h.mass[q], mass_fx(__fsub_rn(z, zmax)));
+            }
+        });
+        __syncthreads();
+        have_hist = true;
+    };
+    if (want_k || want_topp) build_hist(want_topp);
+
+    // top-k stage
     u64 C1 = Cfin;
     u64 n_topk = n_fin;
-    if (rp.top_k >= 1 && rp.top_k < V && (u64)rp.top_k < n_fin) {
+    if (want_k) {
         n_topk = (u64)rp.top_k;
-        C1 = select_by_count<DT>(s, h, c, Cfin, n_topk, 0, 0);
+        int bin; u64 cb, mb;
+        if (find_prefix_bin(s, h, false, want_topp, n_topk, bin, cb, mb))
+            C1 = resolve_cut<DT>(s, h, c, zmax, bin, false, n_topk, cb, Cfin);
+        if (want_topp) build_hist(true);           // (resolving may have reused the histograms)
     }
     out.n_topk = (int32_t)n_topk;
     if (a.dbg_topk_ids && rp.top_k >= 1 && rp.top_k < V && n_topk <= (u64)a.dbg_cap) {
@@ -547,26 +593,50 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         __syncthreads();
     }
     // min-p: a value threshold, never above the top element
-    if (rp.min_p > 0.0f) {
+    if (want_minp) {
         u64 Cm = (u64)minp_key(zmax, rp.min_p) << 32;
         if (Cm > Ctop) Cm = Ctop;
         if (Cm > C1) C1 = Cm;
     }
     // top-p on the mass of the survivors
     u64 C2 = C1;
-    if (rp.top_p < 1.0f) C2 = select_by_mass<DT>(s, h, c, C1, zmax, rp.top_p);
+    if (want_topp) {
+        u64 Sp = 0;
+        if (C1 == Cfin) {
+            u64 lm = 0;
+            for (int q = threadIdx.x; q < HIST_BINS; q += NT) lm += h.mass[q];
+            Sp = block_sum_u64(s, lm);
+        } else {
+            u64 lm = 0;
+            for_each_score<DT>(c, [&](int i, float z) { if (comp_of(key_of(z), i) >= C1) lm += mass_fx(__fsub_rn(z, zmax)); });
+            Sp = block_sum_u64(s, lm);
+        }
+        double t = ceil((double)rp.top_p * (double)Sp);
+        u64 target = t <= 1.0 ? 1ull : (u64)t;
+        if (target > Sp) target = Sp;
+        if (target < 1) target = 1;
+        int bin; u64 cb, mb;
+        if (find_prefix_bin(s, h, true, true, target, bin, cb, mb))
+            C2 = resolve_cut<DT>(s, h, c, zmax, bin, true, target, mb, C1);
+        if (C2 < C1) C2 = C1;
+        have_hist = false;
+    }
 
-    // final pass: mass of the kept set, its size, and the race
+    // final pass: mass of the kept set, its size, and the race.  An element whose score cannot
+    // beat the thread's best even with the luckiest draw (-ln E <= 23) is skipped.
     u64 S_local = 0, n_local = 0, g_best = 0;
+    float best_g = -3.0e38f;
     for_each_score<DT>(c, [&](int i, float z) {
         u64 C = comp_of(key_of(z), i);
         if (C >= C2) {
             float d = __fsub_rn(z, zmax);
             S_local += mass_fx(d);
             n_local += 1;
-            float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, i));
-            u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
-            g_best = G > g_best ? G : g_best;
+            if (d + 23.0f >= best_g) {
+                float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, i));
+                u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
+                if (G > g_best) { g_best = G; best_g = g; }
+            }
         }
     });
     const u64 S_fx = block_sum_u64(s, S_local);
@@ -579,31 +649,32 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     out.logprob = (n_keep == 1) ? 0.0f : (float)(((double)z_tok - (double)zmax) - lnS);
     out.n_keep = (int32_t)n_keep;
 
-    if (a.num_top > 0) {
+    if (want_top_list) {
         // first min(num_top, n_keep) entries of the kept set, in order
-        u64 *list = (u64 *)h.mass;                 // histograms are free again: reuse as two lists
-        u64 *tmp = list + ALBIREO_MAX_NUM_TOP;
-        u64 want = n_keep < (u64)a.num_top ? n_keep : (u64)a.num_top;
-        u64 CN = (want == n_keep) ? C2 : select_by_count<DT>(s, h, c, C2, want, 0, 0);
-        __syncthreads();
-        int n = gather_sorted<DT>(s, c, CN, list, tmp, ALBIREO_MAX_NUM_TOP);
-        for (int j = threadIdx.x; j < a.num_top; j += NT) {
-            int64_t q = (int64_t)b * a.num_top + j;
-            if (j < n) {
-                int id = comp_idx(list[j]);
-                float zj = unkey((uint32_t)(list[j] >> 32));
-                a.out_top_ids[q] = id;
-                a.out_top_logprobs[q] = (float)(((double)zj - (double)zmax) - lnS);
-            } else {
-                a.out_top_ids[q] = -1;
-                a.out_top_logprobs[q] = __uint_as_float(0xFF800000u);
+        const u64 want = n_keep < (u64)a.num_top ? n_keep : (u64)a.num_top;
+        u64 CN = C2;
+        if (want < n_keep) {
+            if (!have_hist) build_hist(false);
+            int bin; u64 cb, mb;
+            if (find_prefix_bin(s, h, false, false, want, bin, cb, mb))
+                CN = resolve_cut<DT>(s, h, c, zmax, bin, false, want, cb, C2);
+        }
+        u64 lo, hi;
+        const int n = gather_if<DT>(s, h, c, [&](u64 C, float) { return C >= CN; }, lo, hi);
+        const int m = n < ALBIREO_MAX_NUM_TOP ? n : ALBIREO_MAX_NUM_TOP;
+        if ((int)threadIdx.x < m) {
+            const u64 C = h.list[threadIdx.x];
+            int rank = 0;
+            for (int q = 0; q < m; ++q) rank += h.list[q] > C;
+            if (rank < a.num_top) {
+                const int64_t o = (int64_t)b * a.num_top + rank;
+                a.out_top_ids[o] = comp_idx(C);
+                a.out_top_logprobs[o] = (n_keep == 1) ? 0.0f : (float)(((double)unkey((uint32_t)(C >> 32)) - (double)zmax) - lnS);
             }
         }
         __syncthreads();
     }
 }
-
-
 
 // ------------------------------------------------------------------ TMA bulk-copy ring
 //
@@ -690,19 +761,6 @@ __device__ __forceinline__ uint32_t warp_incl_scan_u32(uint32_t v) {
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, o); if (lane >= o) v += t; }
     return v;
-}
-
-// block-wide max and min of 32-bit keys (ignore_zero: zeros do not take part in the min)
-__device__ void block_minmax_u32(BlockScratch &s, uint32_t v, uint32_t &mn, uint32_t &mx) {
-    uint32_t wmx = __reduce_max_sync(0xFFFFFFFFu, v);
-    uint32_t wmn = __reduce_min_sync(0xFFFFFFFFu, v ? v : 0xFFFFFFFFu);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) { s.r32a[threadIdx.x >> 5] = wmx; s.r32b[threadIdx.x >> 5] = wmn; }
-    __syncthreads();
-    uint32_t a = s.r32a[0], bmin = s.r32b[0];
-#pragma unroll
-    for (int w = 1; w < NWARPS; ++w) { a = max(a, s.r32a[w]); bmin = min(bmin, s.r32b[w]); }
-    mx = a; mn = bmin;
 }
 
 // One histogram pass over cand[0..n) restricted to keys in [lo, hi]: finds the bin that
@@ -1309,8 +1367,9 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
 // ------------------------------------------------------------------ the kernel
 
 // dynamic shared memory layout (bytes): [candidates (8 KiB) + 512 select bins (2 KiB)]
-// [ring: nstages x 32 KiB][mbarriers][bitmap][coarse][counts]; the general path lays its histograms
-// (cnt 8 KiB, mass 16 KiB) over the first 24 KiB, which it may do because the ring is idle by then
+// [ring: nstages x 32 KiB][mbarriers][bitmap][coarse][counts]; the general path lays its histograms,
+// gather list and search bins (8 + 16 + 16 + 4 KiB) over the first 44 KiB, which it may do because
+// the ring is idle by then
 template <int DT>
 __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -1321,6 +1380,8 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     HistBins h;
     h.cnt = (uint32_t *)smem;
     h.mass = (u64 *)(smem + HIST_BINS * 4);
+    h.list = (u64 *)(smem + HIST_BINS * 12);
+    h.acc = h.list + GL_CAP;
     Ring rg;
     rg.nstages = a.nstages;
     rg.buf = smem + COMMON_BYTES;
