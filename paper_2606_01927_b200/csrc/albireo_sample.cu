@@ -803,10 +803,17 @@ __device__ bool cand_select_pass(BlockScratch &s, const CandSmem &cs, int n, uin
     return true;
 }
 
-// Lower bound t of the k-th largest key in [lo, hi]: count(key >= t) >= k.  One pass.
-__device__ uint32_t cand_select_approx(BlockScratch &s, const CandSmem &cs, int n, int k, uint32_t lo, uint32_t hi) {
-    uint32_t kk = (uint32_t)k; int shift;
-    cand_select_pass(s, cs, n, kk, lo, hi, shift);     // on failure lo is unchanged: keep all
+// Lower bound t of the k-th largest key in [lo, hi]: count(key >= t) >= k.  One pass when the
+// keys spread over the bins; an outlier that stretches the range leaves most keys in one bin, and
+// then up to two more passes narrow that bin.
+__device__ uint32_t cand_select_approx(BlockScratch &s, const CandSmem &cs, int n, int k, uint32_t lo, uint32_t hi, bool zeroed = false) {
+    uint32_t kk = (uint32_t)k; int shift = 1;
+    for (int pass = 0; pass < 3 && shift != 0; ++pass) {
+        if (!cand_select_pass(s, cs, n, kk, lo, hi, shift, zeroed && pass == 0)) break;   // on failure lo is unchanged
+        const uint32_t pop = cs.hist[s.found_digit];
+        __syncthreads();
+        if (pop <= (uint32_t)(k / 4 + 8)) break;
+    }
     return lo;
 }
 // The k-th largest key in [lo, hi] exactly (as many passes as the key range needs).
@@ -1150,8 +1157,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         if (stream_minp && threadIdx.x == 0) s.runmax = kmax;
         // fewer than k valid maxima: the select fails and tau stays at its floor
         if (has_topk && kmax) {
-            uint32_t kk = (uint32_t)k, lo = kmin, hi = kmax; int shift;
-            if (cand_select_pass(s, cs, NT, kk, lo, hi, shift, true)) tau_topk = lo;
+            const uint32_t t = cand_select_approx(s, cs, NT, k, kmin, kmax, true);
+            if (t != kmin || s.found_digit != 0xFFFFFFFFu) tau_topk = t;
         }
         tau_key = tau_topk;
         if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
