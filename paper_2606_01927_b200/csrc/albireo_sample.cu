@@ -200,6 +200,8 @@ struct RowCtx {
     const uint32_t *bitmap;   // V bits (+1 pad word): token appears in the history
     const uint32_t *coarse;   // exclusive popcount prefix per 8 bitmap words
     const uint32_t *counts;   // occurrence count per distinct id, indexed by rank in the bitmap
+    uint32_t n_distinct;      // number of distinct history ids (set bits of the bitmap)
+    int ncoarse;              // entries of `coarse`
 };
 
 __device__ __forceinline__ uint32_t hist_rank(const RowCtx &c, int i) {
@@ -288,48 +290,83 @@ struct HistSmem {
     uint32_t *counts;   // CNT_CAP
 };
 
+// exclusive prefix sum of 32-bit values over the threads of the block (thread order); block total in `total`
+__device__ uint32_t block_exscan_u32(BlockScratch &s, uint32_t v, uint32_t &total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
+    __syncthreads();
+    if (lane == 31) s.r32b[wid] = inc;
+    __syncthreads();
+    uint32_t base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < NWARPS; ++w) { const uint32_t t = s.r32b[w]; base += (w < wid) ? t : 0u; tot += t; }
+    total = tot;
+    return base + inc - v;
+}
+
 // Builds the per-row penalty tables.  Returns false (penalties skipped) if the distinct
 // ids fit neither on chip nor in the caller's workspace.
 __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, const int32_t *ids, int len,
                               uint32_t *ws, int64_t ws_cap, int64_t ws_off) {
     const int V = c.V;
     const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
+    // the first 8 ids of every thread stay in registers for the second sweep
+    constexpr int KEEP = 8;
+    int mine[KEEP];
+#pragma unroll
+    for (int q = 0; q < KEEP; ++q) { const int j = threadIdx.x + q * NT; mine[q] = j < len ? __ldg(ids + j) : -1; }
     for (int w = threadIdx.x; w <= nwords; w += NT) hs.bitmap[w] = 0;
     __syncthreads();
-    for (int j = threadIdx.x; j < len; j += NT) {
+#pragma unroll
+    for (int q = 0; q < KEEP; ++q) { const int t = mine[q]; if (t >= 0 && t < V) atomicOr(&hs.bitmap[t >> 5], 1u << (t & 31)); }
+    for (int j = threadIdx.x + KEEP * NT; j < len; j += NT) {
         int t = __ldg(ids + j);
         if (t >= 0 && t < V) atomicOr(&hs.bitmap[t >> 5], 1u << (t & 31));
     }
     __syncthreads();
     // coarse exclusive prefix: one entry per 8 words; ncoarse <= 2048 for V <= 2^19
-    u64 carry = 0;
+    uint32_t carry = 0;
     for (int base = 0; base < ncoarse; base += NT) {
         int cb = base + threadIdx.x;
         uint32_t pc = 0;
         if (cb < ncoarse) {
             for (int w = cb << 3; w < min(nwords, (cb << 3) + 8); ++w) pc += __popc(hs.bitmap[w]);
         }
-        u64 tot;
-        u64 ex = block_exscan_u64(s, pc, tot);
-        if (cb < ncoarse) hs.coarse[cb] = (uint32_t)(carry + ex);
+        uint32_t tot;
+        uint32_t ex = block_exscan_u32(s, pc, tot);
+        if (cb < ncoarse) hs.coarse[cb] = carry + ex;
         carry += tot;
     }
-    const uint32_t U = (uint32_t)carry;     // distinct valid ids
+    const uint32_t U = carry;               // distinct valid ids
     uint32_t *cnt;
     bool ok = true;
     if (U <= CNT_CAP) cnt = hs.counts;
     else if (ws && ws_off + (int64_t)U <= ws_cap) cnt = ws + ws_off;
     else { cnt = nullptr; ok = false; }
-    c.bitmap = hs.bitmap; c.coarse = hs.coarse; c.counts = cnt;
+    c.bitmap = hs.bitmap; c.coarse = hs.coarse; c.counts = cnt; c.n_distinct = U; c.ncoarse = ncoarse;
     if (!ok) return false;
     for (uint32_t u = threadIdx.x; u < U; u += NT) cnt[u] = 0;
     __syncthreads();
-    for (int j = threadIdx.x; j < len; j += NT) {
+#pragma unroll
+    for (int q = 0; q < KEEP; ++q) { const int t = mine[q]; if (t >= 0 && t < V) atomicAdd(&cnt[hist_rank(c, t)], 1u); }
+    for (int j = threadIdx.x + KEEP * NT; j < len; j += NT) {
         int t = __ldg(ids + j);
         if (t >= 0 && t < V) atomicAdd(&cnt[hist_rank(c, t)], 1u);
     }
     __syncthreads();
     return true;
+}
+
+// token id of the r-th distinct history id (r < n_distinct), i.e. the r-th set bit of the bitmap
+__device__ int hist_id_of_rank(const RowCtx &c, uint32_t r) {
+    int lo = 0, hi = c.ncoarse - 1;            // last coarse block whose prefix is <= r
+    while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (c.coarse[mid] <= r) lo = mid; else hi = mid - 1; }
+    uint32_t rem = r - c.coarse[lo];
+    int w = lo << 3;
+    for (;;) { const uint32_t pc = __popc(c.bitmap[w]); if (rem < pc) break; rem -= pc; ++w; }
+    return (w << 5) + (int)__fns(c.bitmap[w], 0, (int)rem + 1);
 }
 
 // ------------------------------------------------------------------ general path: histogram selection
@@ -1069,6 +1106,43 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
     }
 }
 
+// Starts the stream of a row that the candidate path will take: resets the per-row state, arms the
+// mbarriers and issues the first copies.  Called by the kernel before the history tables are
+// built, so that the first tiles arrive meanwhile; a block barrier must follow before any wait.
+template <int DT>
+__device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c) {
+    typedef Elem<DT> E;
+    if (threadIdx.x != 0) return;
+    const uintptr_t addr = (uintptr_t)c.row;
+    int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
+    if (head > c.V) head = c.V;
+    const int nvec = (c.V - head) / E::PER_VEC;
+    const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
+    const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
+    {
+        s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
+        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
+        for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
+        for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
+        mbar_init(&rg.bar[MAX_STAGES - 1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (ntiles > 0) ring_issue_first(rg, vp, nvec);
+        const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
+        for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
+        s.issued = (uint32_t)npre;
+    }
+}
+
+// which rows the candidate path takes (decided from the row's parameters alone)
+__device__ __forceinline__ bool candidate_eligible(const RowParams &rp, int V) {
+    const int k = rp.greedy ? 1 : rp.top_k;
+    const bool has_topk = rp.greedy || (k >= 1 && k < V);
+    const bool has_minp = !rp.greedy && rp.min_p > 0.0f;
+    if (has_topk && k > KA_MAX) return false;
+    return has_topk || has_minp;
+}
+
 // Returns false if the row must be handled by the general path instead.  On success the
 // results are in `out` for warp 0 only.
 template <int DT>
@@ -1099,19 +1173,6 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
     const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
 
-    if (threadIdx.x == 0) {
-        s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
-        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
-        for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
-        for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
-        mbar_init(&rg.bar[MAX_STAGES - 1], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (ntiles > 0) ring_issue_first(rg, vp, nvec);
-        const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
-        for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
-        s.issued = (uint32_t)npre;
-    }
     cs.hist[threadIdx.x] = 0;
     __syncthreads();
 
@@ -1315,26 +1376,18 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
         }
     }
-    // penalised tokens, straight from the history bitmap
+    // penalised tokens, straight from the history tables: one distinct id per thread and round,
+    // so that a dense head of the vocabulary does not pile up on a few threads
     if (c.has_hist) {
-        const int nwords = (V + 31) >> 5;
-        for (int w = threadIdx.x; w < nwords; w += NT) {
-            uint32_t wbits = c.bitmap[w];
-            if (!wbits) continue;
-            uint32_t r = c.coarse[w >> 3];
-            for (int ww = (w >> 3) << 3; ww < w; ++ww) r += __popc(c.bitmap[ww]);
-            while (wbits) {
-                int bit = __ffs(wbits) - 1;
-                wbits &= wbits - 1;
-                int i = (w << 5) + bit;
-                float x = E::load(c.row, i);
-                uint32_t cntv = c.counts[r++];
-                float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
-                av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cntv)));
-                av = __fsub_rn(av, c.p);
-                uint32_t key = key_of(__fmul_rn(av, c.invT));
-                if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
-            }
+        for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
+            const int i = hist_id_of_rank(c, r);
+            const float x = E::load(c.row, i);
+            const uint32_t cntv = c.counts[r];
+            float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
+            av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cntv)));
+            av = __fsub_rn(av, c.p);
+            const uint32_t key = key_of(__fmul_rn(av, c.invT));
+            if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
         }
     }
     __syncthreads();
@@ -1419,9 +1472,11 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     c.r = a.rep ? a.rep[b] : 1.0f;
     c.p = a.pres ? a.pres[b] : 0.0f;
     c.f = a.freq ? a.freq[b] : 0.0f;
-    c.has_hist = false; c.bitmap = nullptr; c.coarse = nullptr; c.counts = nullptr;
+    c.has_hist = false; c.bitmap = nullptr; c.coarse = nullptr; c.counts = nullptr; c.n_distinct = 0; c.ncoarse = 0;
     if (!(c.r > 0.0f)) out.status |= ALBIREO_ROW_BAD_PARAM;
 
+    const bool try_candidates = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL) && candidate_eligible(rp, V);
+    if (try_candidates) candidate_begin<DT>(s, rg, c);
     if (a.hist_ids && a.hist_off) {
         const int o0 = a.hist_off[b], o1 = a.hist_off[b + 1];
         if (o1 > o0) {
@@ -1446,7 +1501,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     cs.efx = cs.sorted + SORT_MAX;
     cs.gsc = cs.efx + SORT_MAX;
     bool done = false;
-    if (!(a.flags & ALBIREO_FLAG_FORCE_GENERAL)) done = candidate_path<DT>(s, cs, rg, c, rp, a, b, out);
+    if (try_candidates) done = candidate_path<DT>(s, cs, rg, c, rp, a, b, out);
     if (!done) {
         __syncthreads();
         general_path<DT>(s, h, c, rp, a, b, out);
