@@ -106,6 +106,21 @@ __device__ __forceinline__ uint32_t race_word(uint64_t seed, uint32_t R, uint64_
     return wsel == 0 ? c0 : wsel == 1 ? c1 : wsel == 2 ? c2 : c3;
 }
 
+// all four words of the Philox block that serves tokens 4 blk .. 4 blk + 3
+__device__ __forceinline__ uint4 race_block(uint64_t seed, uint32_t R, uint64_t step, uint32_t blk) {
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    uint32_t c0 = blk, c1 = R, c2 = (uint32_t)step, c3 = (uint32_t)(step >> 32);
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        uint32_t h0 = __umulhi(M0, c0), l0 = M0 * c0;
+        uint32_t h1 = __umulhi(M1, c2), l1 = M1 * c2;
+        c0 = h1 ^ c1 ^ k0; c1 = l1; c2 = h0 ^ c3 ^ k1; c3 = l0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
 // -ln(E) for E = -log1p(-v), v = (w + 1/2) 2^-32, in fp32.  The half of the range near
 // v = 1 is evaluated from 1 - v = (~w + 1/2) 2^-32 so both ends keep full relative accuracy.
 __device__ __forceinline__ float neg_log_exp1_f32(uint32_t w) {
@@ -119,6 +134,22 @@ __device__ __forceinline__ float neg_log_exp1_f32(uint32_t w) {
     }
     return -logf(E);
 }
+// The same quantity for the general path, where it is evaluated once per kept element of rows that
+// may keep tens of thousands: branch-free, hardware logarithms.  E = v + v^2/2 + ... for v < 1/4
+// (the small-E end decides the race and keeps full relative accuracy there), E = -ln(1 - v) above;
+// absolute error of the result about 1e-6, inside the band in which the race counts as a near-tie.
+__device__ __forceinline__ float neg_log_exp1_fast(uint32_t w) {
+    const float v = __fmaf_rn((float)w, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+    float p = 1.0f / 12.0f;
+#pragma unroll
+    for (int n = 11; n >= 1; --n) p = __fmaf_rn(p, v, 1.0f / (float)n);
+    const float e_small = p * v;
+    const float omv = __fmaf_rn((float)(~w), 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+    const float e_large = -__logf(omv);
+    const float E = v < 0.25f ? e_small : e_large;
+    return -__logf(E);
+}
+
 __device__ __forceinline__ uint32_t orderable_f32(float g) { return key_of(g); }
 
 // fixed-point mass of an element at distance d = z - zmax <= 0 (deterministic integer sums)
@@ -252,8 +283,12 @@ __device__ __forceinline__ float score_of(const RowCtx &c, int i, float x) {
     return __fmul_rn(a, c.invT);
 }
 
-// Calls fn(i, z_i) for every element of the row (each thread a strided share).
-// 16-byte vector loads over the aligned middle of the row, scalar head and tail.
+__device__ int hist_id_of_rank(const RowCtx &c, uint32_t r);
+
+// Calls fn(i, z_i) exactly once for every element of the row (each thread a share; any order).
+// Unpenalised elements come from 16-byte vector loads over the aligned middle of the row, two
+// loads in flight per thread, plus a scalar head and tail; penalised tokens (whose raw value is not
+// their score) are skipped there and taken from the history tables afterwards.
 template <int DT, class F>
 __device__ __forceinline__ void for_each_score(const RowCtx &c, F &&fn) {
     typedef Elem<DT> E;
@@ -263,23 +298,38 @@ __device__ __forceinline__ void for_each_score(const RowCtx &c, F &&fn) {
     if (head > V) head = V;
     const int nvec = (V - head) / E::PER_VEC;
     const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
-    for (int v = threadIdx.x; v < nvec; v += NT) {
-        const uint4 q = __ldg(vp + v);
-        const int i0 = head + v * E::PER_VEC;
-        uint32_t m = 0;
-        if (c.has_hist) {
-            m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u);
-        }
+    for (int v0 = threadIdx.x; v0 < nvec; v0 += 2 * NT) {
+        const int v1 = v0 + NT;
+        const uint4 q0 = __ldg(vp + v0);
+        const uint4 q1 = v1 < nvec ? __ldg(vp + v1) : q0;
 #pragma unroll
-        for (int e = 0; e < E::PER_VEC; ++e) {
-            float x = E::get(q, e);
-            float a = x;
-            if (m & (1u << e)) a = penalise(c, i0 + e, x);
-            fn(i0 + e, __fmul_rn(a, c.invT));
+        for (int u = 0; u < 2; ++u) {
+            if (u == 1 && v1 >= nvec) break;
+            const uint4 &q = u ? q1 : q0;
+            const int i0 = head + (u ? v1 : v0) * E::PER_VEC;
+            uint32_t m = 0;
+            if (c.has_hist) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+#pragma unroll
+            for (int e = 0; e < E::PER_VEC; ++e)
+                if (!((m >> e) & 1u)) fn(i0 + e, __fmul_rn(E::get(q, e), c.invT));
         }
     }
-    for (int i = threadIdx.x; i < head; i += NT) fn(i, score_of(c, i, E::load(c.row, i)));
-    for (int i = head + nvec * E::PER_VEC + threadIdx.x; i < V; i += NT) fn(i, score_of(c, i, E::load(c.row, i)));
+    const int tail0 = head + nvec * E::PER_VEC;
+    for (int q = threadIdx.x; q < head + (V - tail0); q += NT) {
+        const int i = q < head ? q : tail0 + (q - head);
+        if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
+        fn(i, __fmul_rn(E::load(c.row, i), c.invT));
+    }
+    if (c.has_hist) {
+        for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
+            const int i = hist_id_of_rank(c, r);
+            const float x = E::load(c.row, i);
+            float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
+            av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(c.counts[r])));
+            av = __fsub_rn(av, c.p);
+            fn(i, __fmul_rn(av, c.invT));
+        }
+    }
 }
 
 // ------------------------------------------------------------------ history -> bitmap + counts
@@ -383,11 +433,25 @@ __device__ int hist_id_of_rank(const RowCtx &c, uint32_t r) {
 //   final   the race over the kept set, its mass and its size.
 
 struct HistBins {
-    uint32_t *cnt;   // HIST_BINS
-    u64 *mass;       // HIST_BINS
+    uint32_t *cnt;   // HIST_BINS element counts
+    uint32_t *limb;  // 3 x HIST_BINS: the bins' masses as three 14-bit limbs (32-bit shared-memory
+                     // adds are native and a limb sum cannot overflow for fewer than 2^18 elements;
+                     // a 64-bit add would be a compare-and-swap loop)
     u64 *list;       // GL_CAP composites gathered from the row
     u64 *acc;        // SEL_ACC bins for the on-chip search in the list
 };
+__device__ __forceinline__ void hist_add_mass(const HistBins &h, int q, u64 e) {
+    const uint32_t l0 = (uint32_t)e & 0x3FFFu, l1 = (uint32_t)(e >> 14) & 0x3FFFu, l2 = (uint32_t)(e >> 28);
+    if (l0) atomicAdd(&h.limb[q], l0);
+    if (l1) atomicAdd(&h.limb[HIST_BINS + q], l1);
+    if (l2) atomicAdd(&h.limb[2 * HIST_BINS + q], l2);
+}
+__device__ __forceinline__ u64 hist_mass(const HistBins &h, int q) {
+    return (u64)h.limb[q] + ((u64)h.limb[HIST_BINS + q] << 14) + ((u64)h.limb[2 * HIST_BINS + q] << 28);
+}
+__device__ __forceinline__ void hist_clear(const HistBins &h) {
+    for (int q = threadIdx.x; q < HIST_BINS; q += NT) { h.cnt[q] = 0; h.limb[q] = 0; h.limb[HIST_BINS + q] = 0; h.limb[2 * HIST_BINS + q] = 0; }
+}
 
 constexpr int GL_CAP = 2048;
 constexpr int SEL_ACC = NT;             // one accumulator per thread
@@ -422,6 +486,13 @@ __device__ uint32_t minp_key(float zmax, float min_p) {
     return k < KEY_MIN_FINITE ? KEY_MIN_FINITE : k;
 }
 
+// Mass of an element at distance d = z - zmax <= 0 in 2^40 fixed point, from the hardware
+// exponential (the general path runs it once per element and pass; its relative error of ~2^-21
+// is far inside the logprob tolerance).  Used by every step of the general path alike.
+__device__ __forceinline__ u64 mass_gen(float d) {
+    return d < -28.5f ? 0ull : __float2ull_rn(__expf(d) * FX_SCALE);
+}
+
 // value-linear bin of a finite score z <= zmax; monotone: a larger z never gets a larger bin
 __device__ __forceinline__ int bin_of(float z, float zmax) {
     int b = __float2int_rz(__fsub_rn(zmax, z) * BIN_SCALE);
@@ -436,7 +507,7 @@ __device__ bool find_prefix_bin(BlockScratch &s, const HistBins &h, bool by_mass
     constexpr int PER = HIST_BINS / NT;
     u64 lc = 0, lm = 0;
 #pragma unroll
-    for (int q = 0; q < PER; ++q) { lc += h.cnt[threadIdx.x * PER + q]; if (have_mass) lm += h.mass[threadIdx.x * PER + q]; }
+    for (int q = 0; q < PER; ++q) { lc += h.cnt[threadIdx.x * PER + q]; if (have_mass) lm += hist_mass(h, threadIdx.x * PER + q); }
     u64 totc, totm = 0;
     u64 runc = block_exscan_u64(s, lc, totc);
     u64 runm = have_mass ? block_exscan_u64(s, lm, totm) : 0ull;
@@ -447,7 +518,7 @@ __device__ bool find_prefix_bin(BlockScratch &s, const HistBins &h, bool by_mass
         u64 rc = runc, rm = runm;
         for (int q = 0; q < PER; ++q) {
             const int bq = threadIdx.x * PER + q;
-            const u64 vc = h.cnt[bq], vm = have_mass ? h.mass[bq] : 0ull;
+            const u64 vc = h.cnt[bq], vm = have_mass ? hist_mass(h, bq) : 0ull;
             const u64 r = by_mass ? rm : rc, v = by_mass ? vm : vc;
             if (r < target && target <= r + v) { s.found_digit = (uint32_t)bq; s.found_above = rc; s.bcast[2] = rm; break; }
             rc += vc; rm += vm;
@@ -492,7 +563,7 @@ __device__ u64 list_resolve(BlockScratch &s, const HistBins &h, int n, bool by_m
         for (int i = threadIdx.x; i < n; i += NT) {
             const u64 C = h.list[i];
             if (C >= lo && C <= hi) {
-                const u64 v = by_mass ? mass_fx(__fsub_rn(unkey((uint32_t)(C >> 32)), zmax)) : 1ull;
+                const u64 v = by_mass ? mass_gen(__fsub_rn(unkey((uint32_t)(C >> 32)), zmax)) : 1ull;
                 atomicAdd(&h.acc[(hi - C) >> shift], v);
             }
         }
@@ -528,14 +599,14 @@ __device__ u64 resolve_cut(BlockScratch &s, const HistBins &h, const RowCtx &c, 
     for (int it = 0; it < 8 && n > GL_CAP; ++it) {
         const u64 width = hi - lo;
         const int shift = width < (u64)HIST_BINS ? 0 : bitlen64(width) - 11;
-        for (int q = threadIdx.x; q < HIST_BINS; q += NT) { h.cnt[q] = 0; h.mass[q] = 0; }
+        hist_clear(h);
         __syncthreads();
         for_each_score<DT>(c, [&](int i, float z) {
             const u64 C = comp_of(key_of(z), i);
             if (C >= lo && C <= hi && C >= floorC) {
                 const uint32_t q = (uint32_t)((hi - C) >> shift);
                 atomicAdd(&h.cnt[q], 1u);
-                if (by_mass) atomicAdd(&h.mass[q], mass_fx(__fsub_rn(z, zmax)));
+                if (by_mass) hist_add_mass(h, (int)q, mass_gen(__fsub_rn(z, zmax)));
             }
         });
         __syncthreads();
@@ -564,21 +635,26 @@ template <int DT>
 __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c, const RowParams &rp,
                              const SampleArgs &a, int b, RowOut &out) {
     const int V = c.V;
-    // pass 0: the top element and the number of finite scores
-    u64 best = 0; uint32_t nfin_local = 0;
-    for_each_score<DT>(c, [&](int i, float z) {
-        uint32_t k = key_of(z);
-        u64 C = comp_of(k, i);
-        best = C > best ? C : best;
+    // pass 0: the largest key and the number of finite scores
+    uint32_t kbest = 0, nfin_local = 0;
+    for_each_score<DT>(c, [&](int, float z) {
+        const uint32_t k = key_of(z);
+        kbest = k > kbest ? k : kbest;
         nfin_local += (k >= KEY_MIN_FINITE && k < KEY_POS_INF);
     });
-    const u64 Ctop = block_max_u64(s, best);
+    const uint32_t kmax = (uint32_t)block_max_u64(s, kbest);
     const u64 n_fin = block_sum_u64(s, nfin_local);
-    const float zmax = unkey((uint32_t)(Ctop >> 32));
+    const float zmax = unkey(kmax);
     out.status |= ALBIREO_ROW_GENERAL_PATH;
+    // the first element of the order: the lowest id among the largest keys (one more pass, only when asked for)
+    auto top_id = [&]() -> int {
+        uint32_t best = 0;
+        for_each_score<DT>(c, [&](int i, float z) { if (key_of(z) == kmax) { const uint32_t v = ~(uint32_t)i; best = v > best ? v : best; } });
+        return (int)~(uint32_t)block_max_u64(s, best);
+    };
 
     if (rp.greedy || n_fin <= 1) {
-        out.token = comp_idx(Ctop); out.logprob = 0.0f; out.n_keep = 1; out.n_topk = 1;
+        out.token = top_id(); out.logprob = 0.0f; out.n_keep = 1; out.n_topk = 1;
         if (a.dbg_topk_ids && a.dbg_cap >= 1 && threadIdx.x == 0) a.dbg_topk_ids[(int64_t)b * a.dbg_cap] = out.token;
         if (a.num_top > 0 && threadIdx.x == 0) {
             a.out_top_ids[(int64_t)b * a.num_top] = out.token;
@@ -593,21 +669,22 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const bool want_topp = rp.top_p < 1.0f;
     const bool want_top_list = a.num_top > 0;
     bool have_hist = false;
-    auto build_hist = [&](bool with_mass) {
-        for (int q = threadIdx.x; q < HIST_BINS; q += NT) { h.cnt[q] = 0; h.mass[q] = 0; }
+    auto build_hist = [&](bool with_cnt, bool with_mass) {
+        hist_clear(h);
         __syncthreads();
         for_each_score<DT>(c, [&](int, float z) {
-            const uint32_t k = key_of(z);
-            if (k >= KEY_MIN_FINITE && k < KEY_POS_INF) {
-                const int q = bin_of(z, zmax);
-                atomicAdd(&h.cnt[q], 1u);
-                if (with_mass) atomicAdd(&h.mass[q], mass_fx(__fsub_rn(z, zmax)));
+            const float d = __fsub_rn(zmax, z);               // >= 0 for finite z; inf / NaN otherwise
+            if (d < 3.0e38f) {
+                int q = __float2int_rz(d * BIN_SCALE);
+                q = q > HIST_BINS - 1 ? HIST_BINS - 1 : q;
+                if (with_cnt) atomicAdd(&h.cnt[q], 1u);
+                if (with_mass) { const u64 e = mass_gen(-d); if (e) hist_add_mass(h, q, e); }
             }
         });
         __syncthreads();
-        have_hist = true;
+        have_hist = with_cnt;
     };
-    if (want_k || want_topp) build_hist(want_topp);
+    if (want_k || want_topp) build_hist(want_k, want_topp);
 
     // top-k stage
     u64 C1 = Cfin;
@@ -617,7 +694,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         int bin; u64 cb, mb;
         if (find_prefix_bin(s, h, false, want_topp, n_topk, bin, cb, mb))
             C1 = resolve_cut<DT>(s, h, c, zmax, bin, false, n_topk, cb, Cfin);
-        if (want_topp) build_hist(true);           // (resolving may have reused the histograms)
+        if (want_topp) build_hist(false, true);    // (resolving may have reused the histograms)
     }
     out.n_topk = (int32_t)n_topk;
     if (a.dbg_topk_ids && rp.top_k >= 1 && rp.top_k < V && n_topk <= (u64)a.dbg_cap) {
@@ -632,7 +709,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     // min-p: a value threshold, never above the top element
     if (want_minp) {
         u64 Cm = (u64)minp_key(zmax, rp.min_p) << 32;
-        if (Cm > Ctop) Cm = Ctop;
+        if ((uint32_t)(Cm >> 32) > kmax) Cm = comp_of(kmax, top_id());     // floor above the maximum: the first element alone
         if (Cm > C1) C1 = Cm;
     }
     // top-p on the mass of the survivors
@@ -641,11 +718,12 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         u64 Sp = 0;
         if (C1 == Cfin) {
             u64 lm = 0;
-            for (int q = threadIdx.x; q < HIST_BINS; q += NT) lm += h.mass[q];
+            for (int q = threadIdx.x; q < HIST_BINS; q += NT) lm += hist_mass(h, q);
             Sp = block_sum_u64(s, lm);
         } else {
             u64 lm = 0;
-            for_each_score<DT>(c, [&](int i, float z) { if (comp_of(key_of(z), i) >= C1) lm += mass_fx(__fsub_rn(z, zmax)); });
+            const uint32_t k1 = (uint32_t)(C1 >> 32); const int id1 = comp_idx(C1);
+            for_each_score<DT>(c, [&](int i, float z) { const uint32_t k = key_of(z); if (k > k1 || (k == k1 && i <= id1)) lm += mass_gen(__fsub_rn(z, zmax)); });
             Sp = block_sum_u64(s, lm);
         }
         double t = ceil((double)rp.top_p * (double)Sp);
@@ -661,17 +739,25 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
 
     // final pass: mass of the kept set, its size, and the race.  An element whose score cannot
     // beat the thread's best even with the luckiest draw (-ln E <= 23) is skipped.
-    u64 S_local = 0, n_local = 0, g_best = 0;
+    u64 S_local = 0, g_best = 0;
+    uint32_t n_local = 0;
     float best_g = -3.0e38f;
+    const uint32_t k2 = (uint32_t)(C2 >> 32);
+    const int id2 = comp_idx(C2);
+    uint32_t blk_id = 0xFFFFFFFFu;                       // neighbouring tokens share a Philox block: keep the last one
+    uint4 blk = make_uint4(0, 0, 0, 0);
     for_each_score<DT>(c, [&](int i, float z) {
-        u64 C = comp_of(key_of(z), i);
-        if (C >= C2) {
-            float d = __fsub_rn(z, zmax);
-            S_local += mass_fx(d);
+        const uint32_t k = key_of(z);
+        if (k > k2 || (k == k2 && i <= id2)) {
+            const float d = __fsub_rn(z, zmax);
+            S_local += mass_gen(d);
             n_local += 1;
             if (d + 23.0f >= best_g) {
-                float g = d + neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, i));
-                u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
+                if (((uint32_t)i >> 2) != blk_id) { blk_id = (uint32_t)i >> 2; blk = race_block(rp.seed, rp.R, a.step, blk_id); }
+                const int wsel = i & 3;
+                const uint32_t w = wsel == 0 ? blk.x : wsel == 1 ? blk.y : wsel == 2 ? blk.z : blk.w;
+                const float g = d + neg_log_exp1_fast(w);
+                const u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
                 if (G > g_best) { g_best = G; best_g = g; }
             }
         }
@@ -682,7 +768,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const int tok = comp_idx(G);
     const double lnS = log((double)S_fx) - LN2_40;
     float z_tok = score_of(c, tok, Elem<DT>::load(c.row, tok));
-    out.token = (n_keep == 1) ? comp_idx(Ctop) : tok;
+    out.token = tok;                                   // (a single kept element wins its own race)
     out.logprob = (n_keep == 1) ? 0.0f : (float)(((double)z_tok - (double)zmax) - lnS);
     out.n_keep = (int32_t)n_keep;
 
@@ -691,7 +777,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         const u64 want = n_keep < (u64)a.num_top ? n_keep : (u64)a.num_top;
         u64 CN = C2;
         if (want < n_keep) {
-            if (!have_hist) build_hist(false);
+            if (!have_hist) build_hist(true, false);
             int bin; u64 cb, mb;
             if (find_prefix_bin(s, h, false, false, want, bin, cb, mb))
                 CN = resolve_cut<DT>(s, h, c, zmax, bin, false, want, cb, C2);
@@ -1428,7 +1514,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
 
 // dynamic shared memory layout (bytes): [candidates (8 KiB) + 512 select bins (2 KiB)]
 // [ring: nstages x 32 KiB][mbarriers][bitmap][coarse][counts]; the general path lays its histograms,
-// gather list and search bins (8 + 16 + 16 + 4 KiB) over the first 44 KiB, which it may do because
+// gather list and search bins (8 + 24 + 16 + 4 KiB) over the first 52 KiB, which it may do because
 // the ring is idle by then
 template <int DT>
 __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs a) {
@@ -1439,8 +1525,8 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
 
     HistBins h;
     h.cnt = (uint32_t *)smem;
-    h.mass = (u64 *)(smem + HIST_BINS * 4);
-    h.list = (u64 *)(smem + HIST_BINS * 12);
+    h.limb = (uint32_t *)(smem + HIST_BINS * 4);
+    h.list = (u64 *)(smem + HIST_BINS * 16);
     h.acc = h.list + GL_CAP;
     Ring rg;
     rg.nstages = a.nstages;
