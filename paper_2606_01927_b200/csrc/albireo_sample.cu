@@ -1322,10 +1322,15 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     // with tile t.  Every warp checks s.maint_at before each tile.
     int st = 0;                      // ring stage of the current tile
     uint32_t parity = 0;             // its mbarrier phase
+    const bool early_ckpt = ntiles <= rg.nstages + 2;
+    const uint32_t low_trig = (uint32_t)(has_topk ? 2 * k + 32 : CAND_CAP / 4);
+    bool first_look = true;
     for (int tile = 0; tile < ntiles; ++tile) {
-        // Tile 0 holds the head of the vocabulary and is the densest; right after it the list is
-        // looked at once in any case (a bound from 4x the warm-up sample is much tighter).
-        if ((uint32_t)tile == *(volatile uint32_t *)&s.maint_at || tile == 1) {
+        // Tile 0 holds the head of the vocabulary and is the densest, and a bound from 4x the warm-up
+        // sample is much tighter: if the list is already long after it, it is looked at early --
+        // in short rows at a fixed checkpoint before tile 1, in long rows at a rendezvous that the
+        // last warp to finish tile 0 asks for (see below), which costs rows with a short list nothing.
+        if ((uint32_t)tile == *(volatile uint32_t *)&s.maint_at || (early_ckpt && tile == 1)) {
             __syncthreads();                       // every warp is between tiles: nobody appends
             int n = (int)s.cand_cnt;
             const uint32_t ovf = s.overflow, rmax = s.runmax, tmo = s.timeout;
@@ -1340,7 +1345,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             // make the threshold identical in every thread again
             uint32_t tau_new = tau_topk;
             if (stream_minp && rmax) { seen_max = rmax; uint32_t f = minp_key(unkey(rmax), rp.min_p); tau_new = f > tau_new ? f : tau_new; }
-            const uint32_t trig_now = (tile == 1) ? min(trig, (uint32_t)(has_topk ? 2 * k + 32 : CAND_CAP / 4)) : trig;
+            const uint32_t trig_now = first_look ? min(trig, low_trig) : trig;
+            first_look = false;
             if ((uint32_t)n + 1u >= trig_now) {
                 if (has_topk && n >= k) {
                     uint32_t t = cand_select_approx(s, cs, n, k, tau_topk, rmax);
@@ -1436,6 +1442,10 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             if (old == (uint32_t)(NWARPS - 1)) {   // last warp done with this stage: refill it
                 s.done[st] = 0;
                 __threadfence_block();
+                // every warp has finished tile 0 and none can be past tile nstages (not loaded yet):
+                // a long list is looked at before tile nstages + 1
+                if (tile == 0 && !early_ckpt && *(volatile uint32_t *)&s.cand_cnt + 1u >= low_trig)
+                    atomicMin(&s.maint_at, (uint32_t)(rg.nstages + 1));
                 if (tile + rg.nstages < ntiles && *(volatile uint32_t *)&s.timeout == 0u) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     ring_issue(rg, vp, nvec, tile + rg.nstages, st);
