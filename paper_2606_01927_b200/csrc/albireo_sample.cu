@@ -1548,6 +1548,15 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     hs.coarse = hs.bitmap + (nwords + 1);
     hs.counts = hs.coarse + (ncoarse + 1);
 
+    RowCtx c;
+    c.row = (const char *)a.logits + (size_t)b * (size_t)a.row_stride * Elem<DT>::SIZE;
+    c.V = V;
+    // The ring is started before anything else is read, the row's own parameters included: their
+    // loads and the first tiles then travel together.  A row that turns out to need the general
+    // path waits for these copies before it reuses the shared memory.
+    const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
+    if (ring_started) candidate_begin<DT>(s, rg, c);
+
     RowParams rp;
     rp.T = a.temperature ? a.temperature[b] : 1.0f;
     rp.top_k = a.top_k ? a.top_k[b] : 0;
@@ -1561,9 +1570,6 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; out.status = 0;
     if (rp.T < 0.0f || rp.T != rp.T) out.status |= ALBIREO_ROW_BAD_PARAM;
 
-    RowCtx c;
-    c.row = (const char *)a.logits + (size_t)b * (size_t)a.row_stride * Elem<DT>::SIZE;
-    c.V = V;
     c.invT = rp.greedy ? 1.0f : __fdiv_rn(1.0f, rp.T);
     c.r = a.rep ? a.rep[b] : 1.0f;
     c.p = a.pres ? a.pres[b] : 0.0f;
@@ -1571,8 +1577,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     c.has_hist = false; c.bitmap = nullptr; c.coarse = nullptr; c.counts = nullptr; c.n_distinct = 0; c.ncoarse = 0;
     if (!(c.r > 0.0f)) out.status |= ALBIREO_ROW_BAD_PARAM;
 
-    const bool try_candidates = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL) && candidate_eligible(rp, V);
-    if (try_candidates) candidate_begin<DT>(s, rg, c);
+    const bool try_candidates = ring_started && candidate_eligible(rp, V);
     if (a.hist_ids && a.hist_off) {
         const int o0 = a.hist_off[b], o1 = a.hist_off[b + 1];
         if (o1 > o0) {
@@ -1598,6 +1603,12 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     cs.gsc = cs.efx + SORT_MAX;
     bool done = false;
     if (try_candidates) done = candidate_path<DT>(s, cs, rg, c, rp, a, b, out);
+    else if (ring_started) {
+        // (the barrier above made s.issued visible)
+        bool landed = mbar_wait(&rg.bar[MAX_STAGES - 1], 0u);
+        for (int t = 0; t < (int)s.issued; ++t) landed = mbar_wait(&rg.bar[t], 0u) && landed;
+        if (__syncthreads_or(!landed)) { out.status |= ALBIREO_ROW_TIMEOUT; done = true; }   // the same in every thread
+    }
     if (!done) {
         __syncthreads();
         general_path<DT>(s, h, c, rp, a, b, out);
