@@ -978,22 +978,33 @@ __device__ int cand_compact(BlockScratch &s, const CandSmem &cs, int n, uint32_t
 template <int DT> struct VecTest;
 template <> struct VecTest<ALBIREO_BF16> {
     static __device__ uint32_t raw_threshold(uint32_t tau_key, float invT) {
-        const float tz = unkey(tau_key);
-        const float xg = __fdiv_rn(tz, invT);
-        const uint32_t b16 = __float_as_uint(xg) >> 16;
-        uint32_t k16 = (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
+        // order code of a bf16 pattern (the 16-bit analogue of the score key) and back
         auto bits_of = [](uint32_t kk) { return (kk & 0x8000u) ? (kk & 0x7FFFu) : (~kk & 0xFFFFu); };
         auto passes = [&](uint32_t kk) {
             float x = __uint_as_float(bits_of(kk) << 16);
             return key_of(__fmul_rn(x, invT)) >= tau_key;
         };
-        if (k16 < 0x0080u) k16 = 0x0080u;
-        if (k16 > 0xFF7Fu) k16 = 0xFF7Fu;
-        int it = 0;
-        while (it < 16 && k16 > 0x0080u && passes(k16)) { --k16; ++it; }
-        while (it < 32 && k16 < 0xFF7Fu && !passes(k16)) { ++k16; ++it; }
-        const bool ok = passes(k16) && (k16 == 0x0080u || !passes(k16 - 1));
-        const uint32_t b = ok ? bits_of(k16) : 0xFF80u;     // not settled: let everything through
+        constexpr uint32_t LO = 0x0080u, HI = 0xFF7Fu;         // the finite codes
+        // a guess from an approximate quotient, truncated to bf16: the answer is the guess or a
+        // neighbour, so the four codes around it are tried at once instead of one after another
+        const float xg = __fdividef(unkey(tau_key), invT);
+        const uint32_t b16 = __float_as_uint(xg) >> 16;
+        uint32_t k16 = (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
+        k16 = k16 < LO + 2u ? LO + 2u : (k16 > HI - 1u ? HI - 1u : k16);
+        const bool p0 = passes(k16 - 2u), p1 = passes(k16 - 1u), p2 = passes(k16), p3 = passes(k16 + 1u);
+        uint32_t ans = 0;
+        if (p1 && !p0) ans = k16 - 1u;
+        else if (p2 && !p1) ans = k16;
+        else if (p3 && !p2) ans = k16 + 1u;
+        if (ans == 0) {
+            // not bracketed (an extreme temperature, or the ends of the range): a short walk
+            int it = 0;
+            while (it < 16 && k16 > LO && passes(k16)) { --k16; ++it; }
+            while (it < 32 && k16 < HI && !passes(k16)) { ++k16; ++it; }
+            const bool ok = passes(k16) && (k16 == LO || !passes(k16 - 1u));
+            ans = ok ? k16 : 0u;
+        }
+        const uint32_t b = ans ? bits_of(ans) : 0xFF80u;       // not settled: let everything through
         return b | (b << 16);
     }
     static __device__ __forceinline__ __nv_bfloat162 vmax(const uint4 &q) {
@@ -1195,6 +1206,49 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
 // Starts the stream of a row that the candidate path will take: resets the per-row state, arms the
 // mbarriers and issues the first copies.  Called by the kernel before the history tables are
 // built, so that the first tiles arrive meanwhile; a block barrier must follow before any wait.
+// Threshold of the warm-up: a lower bound of the k-th largest of the block's per-thread maxima `mk`
+// (0: the thread has none), all of which lie in [kmin, kmax].  One pass: the maxima fall into
+// SEL_BINS value-linear bins (a monotone map of the key), each bin also keeps its smallest key; one
+// warp then finds the bin in which the count from the top reaches k and the answer is that bin's
+// smallest key: at least k maxima are not below it.  Returns 0 if there are fewer than k maxima.
+// Needs cs.hist zero and the bin minima 0xFFFFFFFF on entry; contains two barriers, the last at the end.
+__device__ uint32_t warm_select(BlockScratch &s, const CandSmem &cs, uint32_t mk, int k, uint32_t kmin, uint32_t kmax) {
+    uint32_t *binmin = (uint32_t *)(cs.cand + SEL_BINS);
+    const float zmin = unkey(kmin), d = unkey(kmax) - zmin;
+    const float scale = (d > 0.0f && d <= 3.0e38f) ? __fdividef((float)(SEL_BINS - 1), d) : 0.0f;
+    if (mk) {
+        int q = (int)((unkey(mk) - zmin) * scale);
+        q = q < 0 ? 0 : (q > SEL_BINS - 1 ? SEL_BINS - 1 : q);
+        atomicAdd(&cs.hist[q], 1u);
+        atomicMin(&binmin[q], mk);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        constexpr int PER = SEL_BINS / 32;                 // consecutive bins per lane
+        uint32_t cn[PER], sum = 0;
+#pragma unroll
+        for (int q = 0; q < PER; q += 4) {
+            const uint4 v = *(const uint4 *)(cs.hist + PER * lane + q);
+            cn[q] = v.x; cn[q + 1] = v.y; cn[q + 2] = v.z; cn[q + 3] = v.w;
+            sum += v.x + v.y + v.z + v.w;
+        }
+        uint32_t suf = sum;                                // maxima in this lane's bins and above
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_down_sync(0xFFFFFFFFu, suf, o); if (lane + o < 32) suf += t; }
+        uint32_t above = suf - sum;
+        if (lane == 0 && suf < (uint32_t)k) s.found_digit = 0u;
+        if (above < (uint32_t)k && suf >= (uint32_t)k) {   // exactly one lane
+            int q = PER - 1;
+#pragma unroll
+            for (int j = PER - 1; j > 0; --j) { if (above + cn[j] < (uint32_t)k && q == j) { above += cn[j]; q = j - 1; } }
+            s.found_digit = binmin[PER * lane + q];
+        }
+    }
+    __syncthreads();
+    return s.found_digit;
+}
+
 template <int DT>
 __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c) {
     typedef Elem<DT> E;
@@ -1260,6 +1314,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
 
     cs.hist[threadIdx.x] = 0;
+    ((uint32_t *)(cs.cand + SEL_BINS))[threadIdx.x] = 0xFFFFFFFFu;     // warm_select's bin minima
     __syncthreads();
 
     uint32_t tau_topk = KEY_MIN_FINITE;   // the top-k part of the threshold: identical in every thread
@@ -1292,7 +1347,6 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             }
         }
         if (mk < KEY_MIN_FINITE || mk >= KEY_POS_INF) mk = 0;
-        cs.cand[threadIdx.x] = (u64)mk << 32;
         {
             const uint32_t wmx = __reduce_max_sync(0xFFFFFFFFu, mk);
             const uint32_t wmn = __reduce_min_sync(0xFFFFFFFFu, mk ? mk : 0xFFFFFFFFu);
@@ -1304,8 +1358,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         if (stream_minp && threadIdx.x == 0) s.runmax = kmax;
         // fewer than k valid maxima: the select fails and tau stays at its floor
         if (has_topk && kmax) {
-            const uint32_t t = cand_select_approx(s, cs, NT, k, kmin, kmax, true);
-            if (t != kmin || s.found_digit != 0xFFFFFFFFu) tau_topk = t;
+            const uint32_t t = warm_select(s, cs, mk, k, kmin, kmax);
+            if (t > tau_topk) tau_topk = t;
         }
         tau_key = tau_topk;
         if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
