@@ -463,6 +463,7 @@ struct RowParams {
     uint64_t seed;
     uint32_t R;
     bool greedy;
+    double ln_min_p;   // ln(min_p) in fp64, once per row (0 when min-p is off)
 };
 
 struct RowOut {
@@ -470,8 +471,7 @@ struct RowOut {
 };
 
 // smallest fp32 z with (double)z - (double)zmax >= ln(min_p), as an order key
-__device__ uint32_t minp_key(float zmax, float min_p) {
-    const double thr = log((double)min_p);
+__device__ uint32_t minp_key(float zmax, double thr) {
     const double zm = (double)zmax;
     float z = (float)(zm + thr);
     // settle on the exact boundary (a handful of ulp steps at most)
@@ -708,7 +708,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     }
     // min-p: a value threshold, never above the top element
     if (want_minp) {
-        u64 Cm = (u64)minp_key(zmax, rp.min_p) << 32;
+        u64 Cm = (u64)minp_key(zmax, rp.ln_min_p) << 32;
         if ((uint32_t)(Cm >> 32) > kmax) Cm = comp_of(kmax, top_id());     // floor above the maximum: the first element alone
         if (Cm > C1) C1 = Cm;
     }
@@ -1142,7 +1142,7 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         cs.sorted[rank] = C;
         cs.efx[rank] = mass[j];
         cs.gsc[rank] = ((u64)orderable_f32(d + nle[j]) << 32) | (uint32_t)C;
-        in7 = rank < L6 && (!has_minp || ((double)z - (double)zmax >= log((double)rp.min_p)));
+        in7 = rank < L6 && (!has_minp || ((double)z - (double)zmax >= rp.ln_min_p));
     }
     // min-p keeps a prefix of the order, at least one element (the barrier also publishes step 1)
     int L7 = __syncthreads_count(in7);
@@ -1362,7 +1362,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             if (t > tau_topk) tau_topk = t;
         }
         tau_key = tau_topk;
-        if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.min_p); tau_key = f > tau_key ? f : tau_key; }
+        if (stream_minp && kmax) { uint32_t f = minp_key(unkey(kmax), rp.ln_min_p); tau_key = f > tau_key ? f : tau_key; }
         seen_max = kmax;
         thr = T::raw_threshold(tau_key, c.invT);
         if (!(has_topk && kmax)) __syncthreads();       // (the select ends with a barrier of its own)
@@ -1398,7 +1398,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             }
             // make the threshold identical in every thread again
             uint32_t tau_new = tau_topk;
-            if (stream_minp && rmax) { seen_max = rmax; uint32_t f = minp_key(unkey(rmax), rp.min_p); tau_new = f > tau_new ? f : tau_new; }
+            if (stream_minp && rmax) { seen_max = rmax; uint32_t f = minp_key(unkey(rmax), rp.ln_min_p); tau_new = f > tau_new ? f : tau_new; }
             const uint32_t trig_now = first_look ? min(trig, low_trig) : trig;
             first_look = false;
             if ((uint32_t)n + 1u >= trig_now) {
@@ -1421,7 +1421,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             const uint32_t rm = *(volatile uint32_t *)&s.runmax;
             if (rm > seen_max) {
                 seen_max = rm;
-                const uint32_t f = minp_key(unkey(rm), rp.min_p);
+                const uint32_t f = minp_key(unkey(rm), rp.ln_min_p);
                 if (f > tau_key) { tau_key = f; thr = T::raw_threshold(tau_key, c.invT); }
             }
         }
@@ -1555,7 +1555,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         }
         if (n < k && stream_minp) topk_exact_known = false;
     } else {
-        n = cand_compact(s, cs, n, minp_key(unkey(kmax), rp.min_p));
+        n = cand_compact(s, cs, n, minp_key(unkey(kmax), rp.ln_min_p));
         topk_exact_known = false;
     }
     if (n > SORT_MAX || n < 1) return false;
@@ -1619,6 +1619,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     rp.seed = a.seeds ? a.seeds[b] : 0ull;
     rp.R = a.row_base + (uint32_t)b;
     rp.greedy = !(rp.T > 0.0f);
+    rp.ln_min_p = (!rp.greedy && rp.min_p > 0.0f) ? log((double)rp.min_p) : 0.0;
 
     RowOut out;
     out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; out.status = 0;
