@@ -13,7 +13,7 @@
  *
  * The paper fixes none of the arithmetic; the readings taken are listed in the
  * repository's design notes.  In short, per row:
- *   1. widen logits to fp32 (bf16 -> fp32 is exact);
+ *   1. widen logits to fp32 (bf16 -> fp32 and fp16 -> fp32 are exact);
  *   2. count history occurrences per token id (ids outside [0,V) ignored);
  *   3. for tokens with count > 0: a = x>0 ? x/r : x*r ; a -= f*count ; a -= p
  *      (each step one rounded fp32 operation);
@@ -23,7 +23,8 @@
  *   8. top-p: smallest prefix whose mass >= top_p * (mass of the survivors);
  *   9. softmax over the survivors in fp64 -> log-probabilities;
  *  10. exponential race: Philox4x32-10 word per token -> E ~ Exp(1);
- *      token = argmax (z - zmax) - ln E.
+ *      token = argmax (z - zmax) - ln E.  (With pre-generated random numbers, the scheme of
+ *      section 6.2, E is read from a caller-supplied [B, V] fp32 table of Exp(1) variates instead.)
  * Reductions are fp64 in sorted order.  No blocking, fusion or reordering.
  *
  * Nothing here is shared with the CUDA library, and only tests, the smoke check and
@@ -38,6 +39,7 @@
 
 #define ORACLE_F32 0
 #define ORACLE_BF16 1
+#define ORACLE_F16 2      /* IEEE binary16, the precision of the paper's models (section 8.1) */
 
 typedef struct {
     int32_t token;        /* sampled token id                                   */
@@ -73,6 +75,16 @@ static float load_logit(const void *logits, int32_t dtype, int64_t pos)
     if (dtype == ORACLE_BF16) {
         uint16_t h = ((const uint16_t *)logits)[pos];
         return bits_to_f32(((uint32_t)h) << 16);
+    }
+    if (dtype == ORACLE_F16) {
+        /* IEEE binary16 -> fp32, exact: 1 sign, 5 exponent (bias 15), 10 fraction bits */
+        uint16_t h = ((const uint16_t *)logits)[pos];
+        int sign = (h >> 15) & 1, ex = (h >> 10) & 0x1F, fr = h & 0x3FF;
+        float v;
+        if (ex == 0) v = ldexpf((float)fr, -24);                      /* zero and subnormals: fr * 2^-24 */
+        else if (ex == 31) v = fr ? NAN : INFINITY;
+        else v = ldexpf((float)(fr | 0x400), ex - 25);                /* (1024 + fr) * 2^(ex-15-10) */
+        return sign ? -v : v;
     }
     return ((const float *)logits)[pos];
 }
@@ -186,6 +198,7 @@ static int row_scores_and_order(const void *logits, int32_t dtype, int64_t row_p
  */
 static void row_cut_and_draw(const float *z, const sort_item_t *order, int32_t V, int greedy,
                              const row_params_t *rp, uint32_t R, uint64_t step,
+                             const float *exp1_row /* NULL: Philox */,
                              double ln_min_p_shift, double top_p_shift,
                              albireo_oracle_row_t *out, double *e /* scratch [V] */)
 {
@@ -250,7 +263,7 @@ static void row_cut_and_draw(const float *z, const sort_item_t *order, int32_t V
     int32_t best = -1; double gbest = -INFINITY, gsecond = -INFINITY; int32_t jbest = 0;
     for (int32_t j = 0; j < L; ++j) {
         int32_t id = order[j].id;
-        double E = exp1_from_word(race_word(rp->seed, R, step, id));
+        double E = exp1_row ? (double)exp1_row[id] : exp1_from_word(race_word(rp->seed, R, step, id));
         double g = ((double)z[id] - zmax) - log(E);
         if (best < 0 || g > gbest || (g == gbest && id < best)) {
             if (best >= 0) gsecond = gbest;
@@ -294,6 +307,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                           const float *min_p, const float *rep, const float *pres, const float *freq,
                           const int32_t *hist_ids, const int32_t *hist_off,
                           const uint64_t *seeds, uint64_t step, uint32_t row_base,
+                          const float *exp1 /* [B, V] Exp(1) variates, or NULL */,
                           int32_t row_begin, int32_t row_end,
                           albireo_oracle_row_t *rows_out,
                           int32_t topk_cap, int32_t *topk_ids,
@@ -301,7 +315,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                           int32_t num_top, int32_t *top_ids, double *top_logprobs)
 {
     if (!logits || !rows_out || V < 1 || B < 0 || row_begin < 0 || row_end > B) return -1;
-    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return -1;
+    if (dtype != ORACLE_F32 && dtype != ORACLE_BF16 && dtype != ORACLE_F16) return -1;
     float *z = (float *)malloc(sizeof(float) * (size_t)V);
     sort_item_t *order = (sort_item_t *)malloc(sizeof(sort_item_t) * (size_t)V);
     int32_t *counts = (int32_t *)calloc((size_t)V, sizeof(int32_t));
@@ -315,7 +329,8 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
         if (hist_ids && hist_off) { h = hist_ids + hist_off[b]; hl = hist_off[b + 1] - hist_off[b]; }
         int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl, &rp, counts, z, order);
         albireo_oracle_row_t *o = &rows_out[b];
-        row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, 0.0, 0.0, o, e);
+        row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step,
+                         exp1 ? exp1 + (int64_t)b * V : NULL, 0.0, 0.0, o, e);
 
         if (topk_ids) for (int32_t j = 0; j < topk_cap; ++j)
             topk_ids[(int64_t)b * topk_cap + j] = (j < o->n_topk) ? order[j].id : -1;
@@ -350,6 +365,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
                                const float *min_p, const float *rep, const float *pres, const float *freq,
                                const int32_t *hist_ids, const int32_t *hist_off,
                                const uint64_t *seeds, uint64_t step, uint32_t row_base,
+                               const float *exp1,
                                int32_t b, double ln_min_p_shift, double top_p_shift,
                                albireo_oracle_row_t *row_out, int32_t *sorted_ids, float *sorted_z,
                                double *sorted_g)
@@ -365,7 +381,8 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
     const int32_t *h = NULL; int32_t hl = 0;
     if (hist_ids && hist_off) { h = hist_ids + hist_off[b]; hl = hist_off[b + 1] - hist_off[b]; }
     int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl, &rp, counts, z, order);
-    row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step,
+    const float *exp1_row = exp1 ? exp1 + (int64_t)b * V : NULL;
+    row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, exp1_row,
                      ln_min_p_shift, top_p_shift, row_out, e);
     const double zmax = (double)z[order[0].id];
     for (int32_t j = 0; j < V; ++j) {
@@ -373,7 +390,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
         if (sorted_ids) sorted_ids[j] = id;
         if (sorted_z) sorted_z[j] = z[id];
         if (sorted_g) {
-            double E = exp1_from_word(race_word(rp.seed, row_base + (uint32_t)b, step, id));
+            double E = exp1_row ? (double)exp1_row[id] : exp1_from_word(race_word(rp.seed, row_base + (uint32_t)b, step, id));
             sorted_g[j] = ((double)z[id] - zmax) - log(E);
         }
     }

@@ -93,6 +93,7 @@ def _common_args(w):
         _ptr(w.presence_penalty, np.float32), _ptr(w.frequency_penalty, np.float32),
         _ptr(w.history_ids, np.int32), _ptr(w.history_offsets, np.int32),
         _ptr(w.seeds, np.uint64), C.c_uint64(w.step), C.c_uint32(w.row_base),
+        _ptr(getattr(w, "exp1", None), np.float32),
     ]
 
 

@@ -23,6 +23,7 @@ import numpy as np
 
 F32 = 0
 BF16 = 1
+F16 = 2     # IEEE binary16, the precision of the paper's models (§8.1)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -44,7 +45,13 @@ class Workload:
 
     ``None`` for a per-row array means "feature off for every row" (the C-ABI takes
     NULL there).  ``logits`` is float32 ``[B, V]`` for dtype F32 and uint16 bf16 bit
-    patterns ``[B, V]`` for dtype BF16.
+    patterns ``[B, V]`` for dtype BF16 (binary16 bit patterns for dtype F16).
+
+    ``exp1`` switches the draw to pre-generated random numbers (the scheme of §6.2):
+    a float32 ``[B, V]`` table of Exp(1) variates read instead of the counter-based
+    generator.  ``backfill_index`` (int32 ``[B]``, -1 = skip) says where in the next
+    iteration's input-id tensor of ``backfill_len`` entries each row's token goes
+    (early feedback, §5.2).
     """
 
     name: str
@@ -65,6 +72,9 @@ class Workload:
     step: int = 0
     row_base: int = 0
     num_top: int = 0
+    exp1: Optional[np.ndarray] = None
+    backfill_index: Optional[np.ndarray] = None
+    backfill_len: int = 0
     notes: dict = field(default_factory=dict)
 
     @property
@@ -82,6 +92,8 @@ class Workload:
         return int(self.history_ids.size) * 4 + int(self.history_offsets.size) * 4
 
     def logits_f32(self) -> np.ndarray:
+        if self.dtype == F16:
+            return self.logits.view(np.float16).astype(np.float32)
         return self.logits if self.dtype == F32 else bf16_bits_to_f32(self.logits)
 
     def rows(self, lo: int, hi: int) -> "Workload":
@@ -102,7 +114,8 @@ class Workload:
             min_p=cut(self.min_p), repetition_penalty=cut(self.repetition_penalty),
             presence_penalty=cut(self.presence_penalty), frequency_penalty=cut(self.frequency_penalty),
             history_ids=hid, history_offsets=hoff, seeds=cut(self.seeds), step=self.step,
-            row_base=self.row_base + lo, num_top=self.num_top, notes=dict(self.notes))
+            row_base=self.row_base + lo, num_top=self.num_top, exp1=cut(self.exp1),
+            backfill_index=cut(self.backfill_index), backfill_len=self.backfill_len, notes=dict(self.notes))
 
 
 # --------------------------------------------------------------------------- helpers
@@ -297,3 +310,40 @@ def random_small(seed: int, B: int, V: int, dtype: int = F32, *, std=2.0, with_h
         w.presence_penalty = rng.uniform(-0.5, 1.0, size=B).astype(np.float32)
         w.frequency_penalty = rng.uniform(-0.2, 0.5, size=B).astype(np.float32)
     return w
+
+
+def as_f16(w: Workload) -> Workload:
+    """The same workload with its logits rounded to binary16 (stored as uint16 bit patterns)."""
+    import copy
+    out = copy.copy(w)
+    out.name = w.name + "_f16"
+    out.dtype = F16
+    out.logits = np.ascontiguousarray(w.logits_f32().astype(np.float16).view(np.uint16))
+    out.notes = dict(w.notes)
+    return out
+
+
+def with_exp1(w: Workload, seed: int = 7) -> Workload:
+    """The same workload drawing from a pre-generated ``[B, V]`` table of Exp(1) variates."""
+    import copy
+    out = copy.copy(w)
+    out.name = w.name + "_exp1"
+    rng = np.random.Generator(np.random.PCG64(seed))
+    out.exp1 = rng.standard_exponential((w.B, w.V), dtype=np.float32)
+    np.maximum(out.exp1, np.float32(1e-30), out=out.exp1)      # strictly positive: ln E stays finite
+    out.notes = dict(w.notes)
+    return out
+
+
+def with_backfill(w: Workload, seed: int = 11, slack: int = 3) -> Workload:
+    """The same workload with a scattered early-feedback map: row b's token goes to a distinct
+    slot of a ``B + slack`` entry input-id tensor; about one row in eight is skipped (-1)."""
+    import copy
+    out = copy.copy(w)
+    rng = np.random.Generator(np.random.PCG64(seed))
+    out.backfill_len = w.B + slack
+    idx = rng.permutation(out.backfill_len)[: w.B].astype(np.int32)
+    idx[rng.random(w.B) < 0.125] = -1
+    out.backfill_index = idx
+    out.notes = dict(w.notes)
+    return out

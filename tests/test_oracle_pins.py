@@ -458,3 +458,79 @@ def test_acceptable_is_just_the_primary_away_from_boundaries():
         acc = O.acceptable(w, b)
         assert all(a[0] == acc[0][0] and abs(a[1] - acc[0][1]) < 1e-12 for a in acc)
         assert acc[0][0] == int(o.tokens[b])
+
+
+# ------------------------------------------------------------------ fp16 logits and pre-generated Exp(1) variates
+
+def test_f16_widening_exhaustive():
+    # §8.1: the paper's models run in FP16; binary16 -> fp32 is exact, checked against the library cast
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    z = O.row_scores(bits, W.F16)           # T=1, no penalties: z == widened logits
+    ref = bits.view(np.float16).astype(np.float32)
+    ok = ~np.isnan(ref)
+    assert (z.view(np.uint32)[ok] == ref.view(np.uint32)[ok]).all()
+    assert np.isnan(z[~ok]).all()
+
+
+def test_f16_rows_equal_fp32_rows_of_the_same_values():
+    rng = np.random.default_rng(41)
+    x = (rng.standard_normal((6, 300)) * 3).astype(np.float16)
+    w32 = one_row(x.astype(np.float32), T=0.8, top_k=20, top_p=0.9, seed=5)
+    w16 = W.as_f16(w32)
+    assert (w16.logits.view(np.float16) == x).all()
+    a, b = O.sample(w32, kept_cap=20), O.sample(w16, kept_cap=20)
+    assert (a.tokens == b.tokens).all() and (a.kept_ids == b.kept_ids).all()
+    assert (a.logprobs == b.logprobs).all()
+
+
+def test_exp1_table_brute_force_and_forced_winner():
+    # §6.2 (pre-generated random numbers): token = argmax over the kept set of (z - zmax) - ln E[b, t]
+    rng = np.random.default_rng(43)
+    B, V = 5, 12
+    x = (rng.standard_normal((B, V)) * 2).astype(np.float32)
+    w = W.with_exp1(one_row(x, T=1.0, top_k=6, seed=1), seed=3)
+    o = O.sample(w, kept_cap=V)
+    for b in range(B):
+        kept = [i for i in o.kept_ids[b].tolist() if i >= 0]
+        assert len(kept) == 6
+        g = {i: (float(x[b, i]) - float(x[b].max())) - math.log(float(w.exp1[b, i])) for i in kept}
+        assert o.tokens[b] == max(kept, key=lambda i: (g[i], -i))
+    # an almost-zero E for one kept token makes it win; the same E for a token outside the kept set changes nothing
+    for b in range(B):
+        kept = [i for i in o.kept_ids[b].tolist() if i >= 0]
+        out_id = next(i for i in range(V) if i not in kept)
+        w2 = W.with_exp1(one_row(x, T=1.0, top_k=6, seed=1), seed=3)
+        w2.exp1[b, kept[-1]] = np.float32(1e-30)
+        assert O.sample(w2).tokens[b] == kept[-1]
+        w3 = W.with_exp1(one_row(x, T=1.0, top_k=6, seed=1), seed=3)
+        w3.exp1[b, out_id] = np.float32(1e-30)
+        assert O.sample(w3).tokens[b] == o.tokens[b]
+
+
+def test_exp1_table_of_the_philox_variates_reproduces_the_counter_based_draw():
+    rng = np.random.default_rng(47)
+    B, V = 8, 64
+    x = (rng.standard_normal((B, V)) * 2).astype(np.float32)
+    w = one_row(x, T=0.9, top_p=0.95, seed=np.arange(B, dtype=np.uint64) + 100, step=3, row_base=5)
+    ref = O.sample(w)
+    tab = np.empty((B, V), dtype=np.float32)
+    for b in range(B):
+        for t in range(V):
+            tab[b, t] = O.exp1_from_word(O.race_word(100 + b, 5 + b, 3, t))
+    w.exp1 = tab
+    got = O.sample(w)
+    sure = ref.rows["race_gap"] > 1e-5          # fp32 rounding of E moves ln E by < 1e-7
+    assert sure.sum() >= B - 1
+    assert (got.tokens[sure] == ref.tokens[sure]).all()
+    assert np.allclose(got.logprobs[sure], ref.logprobs[sure], atol=0, rtol=0)
+
+
+def test_exp1_table_draw_frequencies():
+    # P(token t) = p_t for independent Exp(1) variates (the exponential race), checked by chi-square
+    V, N = 4, 4000
+    x = np.log(np.array([0.4, 0.3, 0.2, 0.1], dtype=np.float64)).astype(np.float32)
+    w = W.with_exp1(one_row(np.tile(x, (N, 1)), T=1.0), seed=99)
+    tok = O.sample(w).tokens
+    obs = np.bincount(tok, minlength=V)
+    p = np.exp(x.astype(np.float64)); p /= p.sum()
+    assert scipy.stats.chisquare(obs, p * N).pvalue > 1e-4
