@@ -42,7 +42,7 @@ extern "C" {
 
 typedef struct albireo_sampler albireo_sampler_t; /* opaque; created by init, freed by destroy */
 
-enum { ALBIREO_F32 = 0, ALBIREO_BF16 = 1 };
+enum { ALBIREO_F32 = 0, ALBIREO_BF16 = 1, ALBIREO_F16 = 2 /* IEEE binary16: the paper's models are FP16, section 8.1 */ };
 
 enum {
     ALBIREO_OK = 0,
@@ -87,6 +87,31 @@ typedef struct albireo_sample_ext {
                                   active top-k (1 <= k < V, or greedy) whose top-k stage
                                   keeps <= dbg_cap ids                                      */
     uint32_t *out_row_status;  /* [B] device: ALBIREO_ROW_* bits                            */
+
+    /* Pre-generated random numbers (section 6.2: the random numbers of a batch are drawn
+       ahead of the sampling step so that every worker sees the same ones).  When exp1 is
+       not NULL the draw reads E_t = exp1[b * stride + t], an Exp(1) variate per (row,
+       token), instead of running the counter-based generator; seeds and step are then
+       unused.  Only entries of kept tokens are read.  Each E must be a positive finite
+       fp32 (otherwise the row's token is unspecified but in range).                       */
+    const float *exp1;         /* [B, exp1_stride_elems] device, 4-byte aligned, or NULL    */
+    int64_t exp1_stride_elems; /* elements between rows of exp1; 0 means V                  */
+
+    /* Early feedback (section 5.2: the sampler hands each new token straight to the next
+       iteration's input and to the output processor instead of waiting for the host).
+       backfill_ids: the next iteration's input-id tensor; row b's token is stored at
+       backfill_ids[backfill_index[b]] (backfill_index NULL: at [b]); a negative index
+       skips the row, an index >= backfill_len is skipped and sets ALBIREO_ROW_BAD_PARAM.
+       feedback_ring: records (global row id << 32 | token) written with one 8-byte store
+       each at slot (feedback_head + b) mod feedback_cap; the memory may be mapped pinned
+       host memory that the output processor polls (it resets a slot after reading it).
+       Rows whose status has ALBIREO_ROW_TIMEOUT write neither.                             */
+    int32_t *backfill_ids;         /* [backfill_len] device, or NULL                         */
+    const int32_t *backfill_index; /* [B] device, or NULL                                    */
+    int64_t backfill_len;
+    uint64_t *feedback_ring;       /* [feedback_cap] device-visible, 8-byte aligned, or NULL */
+    int64_t feedback_cap;
+    int64_t feedback_head;
 } albireo_sample_ext_t;
 
 /*
@@ -124,7 +149,7 @@ int albireo_sample_init(albireo_sampler_t **out, int32_t device,
  * reaches that point.  `device` of the handle must be current.
  *
  *   logits        [B, V] row-major (row stride = ext->row_stride_elems or V), dtype
- *                 ALBIREO_F32 (float) or ALBIREO_BF16 (bfloat16).  Each value finite or
+ *                 ALBIREO_F32 (float), ALBIREO_BF16 (bfloat16) or ALBIREO_F16 (half).  Each value finite or
  *                 -inf, at least one finite per row (NaN / +inf: result unspecified but
  *                 in range).  Never written.  16-byte aligned rows take the vector path;
  *                 any element-aligned pointer/stride is accepted.

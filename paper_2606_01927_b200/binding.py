@@ -18,6 +18,14 @@ from . import _build
 
 F32 = 0
 BF16 = 1
+F16 = 2
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    try:
+        return {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}[t.dtype]
+    except KeyError:
+        raise ValueError("logits must be float32, bfloat16 or float16") from None
 OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED = 0, -1, -2, -3, -4
 ROW_GENERAL_PATH, ROW_BAD_PARAM, ROW_HISTORY_OVERFLOW, ROW_TIMEOUT = 1, 2, 4, 8
 FLAG_FORCE_GENERAL = 1
@@ -39,6 +47,9 @@ class SampleExt(C.Structure):
         ("out_top_ids", C.c_void_p), ("out_top_logprobs", C.c_void_p),
         ("out_num_kept", C.c_void_p), ("out_num_topk", C.c_void_p),
         ("dbg_cap", C.c_int32), ("dbg_topk_ids", C.c_void_p), ("out_row_status", C.c_void_p),
+        ("exp1", C.c_void_p), ("exp1_stride_elems", C.c_int64),
+        ("backfill_ids", C.c_void_p), ("backfill_index", C.c_void_p), ("backfill_len", C.c_int64),
+        ("feedback_ring", C.c_void_p), ("feedback_cap", C.c_int64), ("feedback_head", C.c_int64),
     ]
 
 
@@ -188,18 +199,20 @@ class Sampler:
                        history_ids=None, history_offsets=None, seeds=None, step: int = 0,
                        out_tokens=None, out_logprobs=None, stream: Optional[torch.cuda.Stream] = None,
                        row_base: int = 0, num_top: int = 0, want_counts=False, dbg_cap: int = 0,
-                       want_status=False, flags: int = 0, B: Optional[int] = None, V: Optional[int] = None) -> SampleOutputs:
-        """Device-resident call: all tensors on ``self.device``; asynchronous on ``stream``."""
+                       want_status=False, flags: int = 0, B: Optional[int] = None, V: Optional[int] = None,
+                       exp1: Optional[torch.Tensor] = None, backfill_ids: Optional[torch.Tensor] = None,
+                       backfill_index: Optional[torch.Tensor] = None, feedback_ring: Optional[torch.Tensor] = None,
+                       feedback_head: int = 0) -> SampleOutputs:
+        """Device-resident call: all tensors on ``self.device``; asynchronous on ``stream``.
+
+        ``exp1`` (float32 ``[B, V]``) replaces the counter-based draw by pre-generated Exp(1)
+        variates; ``backfill_ids`` / ``backfill_index`` (int32) and ``feedback_ring`` (int64,
+        device or pinned host memory) are the early-feedback targets."""
         if logits.dim() != 2 or logits.stride(1) != 1:
             raise ValueError("logits must be [B, V] with unit stride along V")
         B = logits.shape[0] if B is None else B
         V = logits.shape[1] if V is None else V
-        if logits.dtype == torch.float32:
-            dt = F32
-        elif logits.dtype == torch.bfloat16:
-            dt = BF16
-        else:
-            raise ValueError("logits must be float32 or bfloat16")
+        dt = _dtype_code(logits)
         dev = logits.device
         if out_tokens is None:
             out_tokens = torch.empty(B, dtype=torch.int32, device=dev)
@@ -209,6 +222,21 @@ class Sampler:
         ext, extra = self._ext(B, "cuda", dev, row_base=row_base, row_stride=0 if row_stride == V else row_stride,
                                num_top=num_top, want_counts=want_counts, dbg_cap=dbg_cap,
                                want_status=want_status, flags=flags)
+        if exp1 is not None:
+            if exp1.dtype != torch.float32 or exp1.dim() != 2 or exp1.stride(1) != 1 or exp1.device != dev:
+                raise ValueError("exp1 must be a float32 [B, V] tensor on the logits' device")
+            ext.exp1 = exp1.data_ptr()
+            ext.exp1_stride_elems = 0 if (B <= 1 or exp1.stride(0) == V) else exp1.stride(0)
+        if backfill_ids is not None:
+            ext.backfill_ids = _dp(backfill_ids, torch.int32, "cuda")
+            ext.backfill_index = _dp(backfill_index, torch.int32, "cuda")
+            ext.backfill_len = backfill_ids.numel()
+        if feedback_ring is not None:
+            if feedback_ring.dtype != torch.int64 or not feedback_ring.is_contiguous():
+                raise ValueError("feedback_ring must be a contiguous int64 tensor (device, or pinned host memory)")
+            ext.feedback_ring = feedback_ring.data_ptr()
+            ext.feedback_cap = feedback_ring.numel()
+            ext.feedback_head = feedback_head
         st = torch.cuda.current_stream(dev) if stream is None else stream
         f32, i32 = torch.float32, torch.int32
         with torch.cuda.device(dev):
@@ -232,9 +260,7 @@ class Sampler:
                             flags: int = 0) -> SampleOutputs:
         """Host-buffer call (CPU tensors, ideally pinned): copies in, samples, copies out, waits."""
         B, V = logits.shape
-        dt = F32 if logits.dtype == torch.float32 else BF16
-        if logits.dtype not in (torch.float32, torch.bfloat16):
-            raise ValueError("logits must be float32 or bfloat16")
+        dt = _dtype_code(logits)
         if out_tokens is None:
             out_tokens = torch.empty(B, dtype=torch.int32, pin_memory=True)
         if out_logprobs is None:
@@ -267,9 +293,7 @@ def albireo_sample_fixed_scratch(logits: torch.Tensor, *, temperature=None, top_
     fixed scratch array is used).  The output tensors created here when none are passed are a
     convenience of this Python wrapper; the C entry point itself allocates nothing."""
     B, V = logits.shape
-    dt = F32 if logits.dtype == torch.float32 else BF16
-    if logits.dtype not in (torch.float32, torch.bfloat16):
-        raise ValueError("logits must be float32 or bfloat16")
+    dt = _dtype_code(logits)
     dev = logits.device
     if out_tokens is None:
         out_tokens = torch.empty(B, dtype=torch.int32, device=dev)
@@ -319,9 +343,17 @@ def workload_tensors(w, device, pinned: bool = False) -> dict:
         hid = np.zeros(1, dtype=np.int32)      # an empty CSR still needs a non-NULL pointer
     if w.dtype == F32:
         logits = conv(w.logits)
+    elif w.dtype == F16:
+        logits = conv(w.logits.view(np.int16), torch.float16)
     else:
         logits = conv(w.logits.view(np.int16), torch.bfloat16)
+    extra = {}
+    if getattr(w, "exp1", None) is not None:
+        extra["exp1"] = conv(w.exp1)
+    if getattr(w, "backfill_index", None) is not None:
+        extra["backfill_index"] = conv(w.backfill_index)
     return dict(
+        **extra,
         logits=logits, temperature=conv(w.temperature), top_k=conv(w.top_k), top_p=conv(w.top_p),
         min_p=conv(w.min_p), repetition_penalty=conv(w.repetition_penalty),
         presence_penalty=conv(w.presence_penalty), frequency_penalty=conv(w.frequency_penalty),

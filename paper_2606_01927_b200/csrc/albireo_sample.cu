@@ -18,6 +18,7 @@
 
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdio.h>
@@ -72,6 +73,13 @@ struct SampleArgs {
     int32_t *dbg_topk_ids;
     uint32_t *out_row_status;
     int32_t nstages;            // ring depth chosen by the host for this launch
+    const float *exp1;          // pre-generated Exp(1) variates [B, exp1_stride], or null: counter-based draw
+    int64_t exp1_stride;
+    int32_t *backfill_ids;      // early feedback: next iteration's input ids, or null
+    const int32_t *backfill_index;
+    int64_t backfill_len;
+    unsigned long long *feedback_ring;   // (row id << 32 | token) records for the output processor, or null
+    int64_t feedback_cap, feedback_head;
     uint32_t *ws_counts;        // global scratch for history counts of rows with many distinct ids
     int64_t ws_counts_cap;      // entries
 };
@@ -274,6 +282,20 @@ template <> struct Elem<ALBIREO_BF16> {
     static __device__ __forceinline__ float get(const uint4 &q, int e) {
         uint32_t w = (e >> 1) == 0 ? q.x : (e >> 1) == 1 ? q.y : (e >> 1) == 2 ? q.z : q.w;
         return __uint_as_float((e & 1) ? (w & 0xFFFF0000u) : (w << 16));
+    }
+};
+
+template <> struct Elem<ALBIREO_F16> {
+    static constexpr int SIZE = 2, PER_VEC = 8;
+    static __device__ __forceinline__ float load(const void *row, int i) {
+        return __half2float(__ushort_as_half(__ldg((const unsigned short *)row + i)));
+    }
+    static __device__ __forceinline__ float load_plain(const void *p, int i) {
+        return __half2float(__ushort_as_half(((const unsigned short *)p)[i]));
+    }
+    static __device__ __forceinline__ float get(const uint4 &q, int e) {
+        uint32_t w = (e >> 1) == 0 ? q.x : (e >> 1) == 1 ? q.y : (e >> 1) == 2 ? q.z : q.w;
+        return __half2float(__ushort_as_half((unsigned short)((e & 1) ? (w >> 16) : (w & 0xFFFFu))));
     }
 };
 
@@ -591,7 +613,7 @@ __device__ u64 list_resolve(BlockScratch &s, const HistBins &h, int n, bool by_m
 // `bin` and that `before` of the total lies in the bins ahead of it.
 template <int DT>
 __device__ u64 resolve_cut(BlockScratch &s, const HistBins &h, const RowCtx &c, float zmax, int bin, bool by_mass,
-                           u64 target, u64 before, u64 floorC) {
+                           u64 target, u64 before, u64 floorC, bool &hist_clobbered) {
     u64 rel = target - before;
     u64 lo, hi;
     int n = gather_if<DT>(s, h, c, [&](u64 C, float z) { return C >= floorC && (C >> 32) < KEY_POS_INF && bin_of(z, zmax) == bin; }, lo, hi);
@@ -599,6 +621,7 @@ __device__ u64 resolve_cut(BlockScratch &s, const HistBins &h, const RowCtx &c, 
     for (int it = 0; it < 8 && n > GL_CAP; ++it) {
         const u64 width = hi - lo;
         const int shift = width < (u64)HIST_BINS ? 0 : bitlen64(width) - 11;
+        hist_clobbered = true;                               // the value histograms are overwritten
         hist_clear(h);
         __syncthreads();
         for_each_score<DT>(c, [&](int i, float z) {
@@ -668,7 +691,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const bool want_minp = rp.min_p > 0.0f;
     const bool want_topp = rp.top_p < 1.0f;
     const bool want_top_list = a.num_top > 0;
-    bool have_hist = false;
+    bool have_hist = false, have_mass = false;           // which value histograms are current
     auto build_hist = [&](bool with_cnt, bool with_mass) {
         hist_clear(h);
         __syncthreads();
@@ -682,7 +705,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
             }
         });
         __syncthreads();
-        have_hist = with_cnt;
+        have_hist = with_cnt; have_mass = with_mass;
     };
     if (want_k || want_topp) build_hist(want_k, want_topp);
 
@@ -692,9 +715,11 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     if (want_k) {
         n_topk = (u64)rp.top_k;
         int bin; u64 cb, mb;
-        if (find_prefix_bin(s, h, false, want_topp, n_topk, bin, cb, mb))
-            C1 = resolve_cut<DT>(s, h, c, zmax, bin, false, n_topk, cb, Cfin);
-        if (want_topp) build_hist(false, true);    // (resolving may have reused the histograms)
+        const bool find_ok = find_prefix_bin(s, h, false, want_topp, n_topk, bin, cb, mb);
+        bool clobbered = false;
+        if (find_ok) C1 = resolve_cut<DT>(s, h, c, zmax, bin, false, n_topk, cb, Cfin, clobbered);
+        if (clobbered) have_hist = have_mass = false;
+        if (want_topp && !have_mass) build_hist(false, true);
     }
     out.n_topk = (int32_t)n_topk;
     if (a.dbg_topk_ids && rp.top_k >= 1 && rp.top_k < V && n_topk <= (u64)a.dbg_cap) {
@@ -731,14 +756,15 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         if (target > Sp) target = Sp;
         if (target < 1) target = 1;
         int bin; u64 cb, mb;
+        bool clobbered = false;
         if (find_prefix_bin(s, h, true, true, target, bin, cb, mb))
-            C2 = resolve_cut<DT>(s, h, c, zmax, bin, true, target, mb, C1);
+            C2 = resolve_cut<DT>(s, h, c, zmax, bin, true, target, mb, C1, clobbered);
         if (C2 < C1) C2 = C1;
-        have_hist = false;
+        if (clobbered) have_hist = have_mass = false;
     }
 
     // final pass: mass of the kept set, its size, and the race.  An element whose score cannot
-    // beat the thread's best even with the luckiest draw (-ln E <= 23) is skipped.
+    // beat the thread's best even with the luckiest draw (-ln E <= 23 for the generator's words) is skipped.
     u64 S_local = 0, g_best = 0;
     uint32_t n_local = 0;
     float best_g = -3.0e38f;
@@ -746,17 +772,24 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const int id2 = comp_idx(C2);
     uint32_t blk_id = 0xFFFFFFFFu;                       // neighbouring tokens share a Philox block: keep the last one
     uint4 blk = make_uint4(0, 0, 0, 0);
+    const float *exp1_row = a.exp1 ? a.exp1 + (int64_t)b * a.exp1_stride : nullptr;
+    const float luck = exp1_row ? 104.0f : 23.0f;        // largest -ln E: a table may hold any positive fp32
     for_each_score<DT>(c, [&](int i, float z) {
         const uint32_t k = key_of(z);
         if (k > k2 || (k == k2 && i <= id2)) {
             const float d = __fsub_rn(z, zmax);
             S_local += mass_gen(d);
             n_local += 1;
-            if (d + 23.0f >= best_g) {
-                if (((uint32_t)i >> 2) != blk_id) { blk_id = (uint32_t)i >> 2; blk = race_block(rp.seed, rp.R, a.step, blk_id); }
-                const int wsel = i & 3;
-                const uint32_t w = wsel == 0 ? blk.x : wsel == 1 ? blk.y : wsel == 2 ? blk.z : blk.w;
-                const float g = d + neg_log_exp1_fast(w);
+            if (d + luck >= best_g) {
+                float nle;
+                if (exp1_row) nle = -logf(__ldg(exp1_row + i));
+                else {
+                    if (((uint32_t)i >> 2) != blk_id) { blk_id = (uint32_t)i >> 2; blk = race_block(rp.seed, rp.R, a.step, blk_id); }
+                    const int wsel = i & 3;
+                    const uint32_t w = wsel == 0 ? blk.x : wsel == 1 ? blk.y : wsel == 2 ? blk.z : blk.w;
+                    nle = neg_log_exp1_fast(w);
+                }
+                const float g = d + nle;
                 const u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
                 if (G > g_best) { g_best = G; best_g = g; }
             }
@@ -779,8 +812,9 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         if (want < n_keep) {
             if (!have_hist) build_hist(true, false);
             int bin; u64 cb, mb;
+            bool clobbered = false;
             if (find_prefix_bin(s, h, false, false, want, bin, cb, mb))
-                CN = resolve_cut<DT>(s, h, c, zmax, bin, false, want, cb, C2);
+                CN = resolve_cut<DT>(s, h, c, zmax, bin, false, want, cb, C2, clobbered);
         }
         u64 lo, hi;
         const int n = gather_if<DT>(s, h, c, [&](u64 C, float) { return C >= CN; }, lo, hi);
@@ -973,22 +1007,37 @@ __device__ int cand_compact(BlockScratch &s, const CandSmem &cs, int n, uint32_t
 }
 
 // Vector pre-test per dtype, in the domain the test runs in.
-// bf16: raw logits; the threshold is the smallest raw bf16 whose score has key >= tau
-// (packed twice).  fp32: scores; the threshold is unkey(tau).
+// 16-bit types: raw logits; the threshold is the smallest raw value whose score has key >= tau
+// (packed twice).  x -> fl32(x * invT) is increasing, strictly so on distinct 16-bit values unless
+// the product leaves the fp32 range, so a compare of raw values is a superset of the key test.
+// fp32: scores; the threshold is unkey(tau).
+struct Bf16Packed {
+    typedef __nv_bfloat162 H2;
+    static constexpr uint32_t LO = 0x0080u, HI = 0xFF7Fu, NEG_INF = 0xFF80u;    // order codes of the finite range; -inf pattern
+    static __device__ __forceinline__ float widen(uint32_t bits) { return __uint_as_float(bits << 16); }
+    static __device__ __forceinline__ uint32_t truncate(float x) { return __float_as_uint(x) >> 16; }
+};
+struct F16Packed {
+    typedef __half2 H2;
+    static constexpr uint32_t LO = 0x0400u, HI = 0xFBFFu, NEG_INF = 0xFC00u;
+    static __device__ __forceinline__ float widen(uint32_t bits) { return __half2float(__ushort_as_half((unsigned short)bits)); }
+    static __device__ __forceinline__ uint32_t truncate(float x) { return __half_as_ushort(__float2half_rz(x)); }
+};
 template <int DT> struct VecTest;
-template <> struct VecTest<ALBIREO_BF16> {
+template <class P> struct VecTest16 {
+    typedef typename P::H2 H2;
     static __device__ uint32_t raw_threshold(uint32_t tau_key, float invT) {
-        // order code of a bf16 pattern (the 16-bit analogue of the score key) and back
+        // order code of a 16-bit pattern (the analogue of the score key) and back
         auto bits_of = [](uint32_t kk) { return (kk & 0x8000u) ? (kk & 0x7FFFu) : (~kk & 0xFFFFu); };
         auto passes = [&](uint32_t kk) {
-            float x = __uint_as_float(bits_of(kk) << 16);
+            float x = P::widen(bits_of(kk));
             return key_of(__fmul_rn(x, invT)) >= tau_key;
         };
-        constexpr uint32_t LO = 0x0080u, HI = 0xFF7Fu;         // the finite codes
-        // a guess from an approximate quotient, truncated to bf16: the answer is the guess or a
+        constexpr uint32_t LO = P::LO, HI = P::HI;             // the finite codes
+        // a guess from an approximate quotient, truncated to 16 bits: the answer is the guess or a
         // neighbour, so the four codes around it are tried at once instead of one after another
         const float xg = __fdividef(unkey(tau_key), invT);
-        const uint32_t b16 = __float_as_uint(xg) >> 16;
+        const uint32_t b16 = P::truncate(xg) & 0xFFFFu;
         uint32_t k16 = (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
         k16 = k16 < LO + 2u ? LO + 2u : (k16 > HI - 1u ? HI - 1u : k16);
         const bool p0 = passes(k16 - 2u), p1 = passes(k16 - 1u), p2 = passes(k16), p3 = passes(k16 + 1u);
@@ -1004,40 +1053,42 @@ template <> struct VecTest<ALBIREO_BF16> {
             const bool ok = passes(k16) && (k16 == LO || !passes(k16 - 1u));
             ans = ok ? k16 : 0u;
         }
-        const uint32_t b = ans ? bits_of(ans) : 0xFF80u;       // not settled: let everything through
+        const uint32_t b = ans ? bits_of(ans) : P::NEG_INF;    // not settled: let everything through
         return b | (b << 16);
     }
-    static __device__ __forceinline__ __nv_bfloat162 vmax(const uint4 &q) {
-        __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x), *reinterpret_cast<const __nv_bfloat162 *>(&q.y));
-        __nv_bfloat162 b2 = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&q.z), *reinterpret_cast<const __nv_bfloat162 *>(&q.w));
+    static __device__ __forceinline__ H2 vmax(const uint4 &q) {
+        H2 a = __hmax2(*reinterpret_cast<const H2 *>(&q.x), *reinterpret_cast<const H2 *>(&q.y));
+        H2 b2 = __hmax2(*reinterpret_cast<const H2 *>(&q.z), *reinterpret_cast<const H2 *>(&q.w));
         return __hmax2(a, b2);
     }
     static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
-        return __hge2_mask(vmax(q), *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
+        return __hge2_mask(vmax(q), *reinterpret_cast<const H2 *>(&thr)) != 0u;
     }
     static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float) {
-        __nv_bfloat162 m = vmax(q[0]);
+        H2 m = vmax(q[0]);
 #pragma unroll
         for (int u = 1; u < TILE_VECS; ++u) m = __hmax2(m, vmax(q[u]));
-        return __hge2_mask(m, *reinterpret_cast<const __nv_bfloat162 *>(&thr)) != 0u;
+        return __hge2_mask(m, *reinterpret_cast<const H2 *>(&thr)) != 0u;
     }
     // bit e set: raw element e >= the raw threshold (a superset of "score key >= tau")
     static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float) {
-        const __nv_bfloat162 t2 = *reinterpret_cast<const __nv_bfloat162 *>(&thr);
-        const uint32_t r0 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.x), t2);
-        const uint32_t r1 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.y), t2);
-        const uint32_t r2 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.z), t2);
-        const uint32_t r3 = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&q.w), t2);
+        const H2 t2 = *reinterpret_cast<const H2 *>(&thr);
+        const uint32_t r0 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.x), t2);
+        const uint32_t r1 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.y), t2);
+        const uint32_t r2 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.z), t2);
+        const uint32_t r3 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.w), t2);
         return ((r0 & 1u) | ((r0 >> 15) & 2u)) | (((r1 & 1u) | ((r1 >> 15) & 2u)) << 2) |
                (((r2 & 1u) | ((r2 >> 15) & 2u)) << 4) | (((r3 & 1u) | ((r3 >> 15) & 2u)) << 6);
     }
     // key of the score of the vector's largest element (an element of the row)
     static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) {
-        __nv_bfloat162 m = vmax(q);
+        H2 m = vmax(q);
         return key_of(__fmul_rn(fmaxf(__low2float(m), __high2float(m)), invT));
     }
-    static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
+    static __device__ __forceinline__ uint4 fill() { const uint32_t f = P::NEG_INF | (P::NEG_INF << 16); return make_uint4(f, f, f, f); }
 };
+template <> struct VecTest<ALBIREO_BF16> : VecTest16<Bf16Packed> {};
+template <> struct VecTest<ALBIREO_F16> : VecTest16<F16Packed> {};
 template <> struct VecTest<ALBIREO_F32> {
     static __device__ uint32_t raw_threshold(uint32_t tau_key, float) { return __float_as_uint(unkey(tau_key)); }
     static __device__ __forceinline__ float vmaxz(const uint4 &q, float invT) {
@@ -1129,7 +1180,8 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         const int t = dense_ok ? (int)threadIdx.x - dstart : (part == 0 ? j : -1);
         if (t >= 0 && t < n) {
             const u64 Ct = cs.cand[t];
-            nle[t] = neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, comp_idx(Ct)));
+            nle[t] = a.exp1 ? -logf(__ldg(a.exp1 + (int64_t)b * a.exp1_stride + comp_idx(Ct)))
+                            : neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, comp_idx(Ct)));
             mass[t] = mass_fx(__fsub_rn(unkey((uint32_t)(Ct >> 32)), zmax));
         }
     }
@@ -1674,6 +1726,21 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
         a.out_logprobs[b] = out.logprob;
         if (a.out_num_kept) a.out_num_kept[b] = out.n_keep;
         if (a.out_num_topk) a.out_num_topk[b] = out.n_topk;
+        // early feedback (section 5.2): the token goes straight into the next iteration's input ids
+        // and to the output processor's ring, without waiting for a host round trip
+        const bool have_token = !(out.status & ALBIREO_ROW_TIMEOUT);
+        if (a.backfill_ids && have_token) {
+            const int64_t slot = a.backfill_index ? (int64_t)a.backfill_index[b] : (int64_t)b;
+            if (slot >= 0) {
+                if (slot < a.backfill_len) a.backfill_ids[slot] = out.token;
+                else out.status |= ALBIREO_ROW_BAD_PARAM;
+            }
+        }
+        if (a.feedback_ring && have_token) {
+            const int64_t slot = (a.feedback_head + b) % a.feedback_cap;
+            const unsigned long long rec = ((unsigned long long)(a.row_base + (uint32_t)b) << 32) | (uint32_t)out.token;
+            *(volatile unsigned long long *)(a.feedback_ring + slot) = rec;      // one 8-byte store
+        }
         if (a.out_row_status) a.out_row_status[b] = out.status;
     }
 }
@@ -1698,6 +1765,67 @@ size_t smem_bytes_for(int V, bool with_history, int nstages) {
 }
 
 constexpr size_t WS_HEADER = 256;
+
+// Checks the optional arguments and copies them into the launch arguments; on failure *why says what.
+int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, const char **why) {
+    (void)B;
+    if (ext->struct_size != sizeof(albireo_sample_ext_t)) { *why = "ext->struct_size mismatch"; return ALBIREO_EINVAL; }
+    if (ext->row_stride_elems != 0) {
+        if (ext->row_stride_elems < V) { *why = "row stride smaller than V"; return ALBIREO_EINVAL; }
+        a.row_stride = ext->row_stride_elems;
+    }
+    a.row_base = ext->row_base; a.flags = ext->flags;
+    if (ext->num_top < 0 || ext->num_top > ALBIREO_MAX_NUM_TOP) { *why = "num_top out of range"; return ALBIREO_EUNSUPPORTED; }
+    if (ext->num_top > 0 && (!ext->out_top_ids || !ext->out_top_logprobs)) { *why = "num_top > 0 needs both top-N outputs"; return ALBIREO_EINVAL; }
+    a.num_top = ext->num_top; a.out_top_ids = ext->out_top_ids; a.out_top_logprobs = ext->out_top_logprobs;
+    a.out_num_kept = ext->out_num_kept; a.out_num_topk = ext->out_num_topk;
+    if (ext->dbg_cap < 0 || (ext->dbg_cap > 0 && !ext->dbg_topk_ids)) { *why = "bad dbg_cap / dbg_topk_ids"; return ALBIREO_EINVAL; }
+    a.dbg_cap = ext->dbg_topk_ids ? ext->dbg_cap : 0;
+    a.dbg_topk_ids = ext->dbg_cap > 0 ? ext->dbg_topk_ids : nullptr;
+    a.out_row_status = ext->out_row_status;
+    if (ext->exp1) {
+        if (ext->exp1_stride_elems != 0 && ext->exp1_stride_elems < V) { *why = "exp1 row stride smaller than V"; return ALBIREO_EINVAL; }
+        if ((uintptr_t)ext->exp1 % 4) { *why = "exp1 not 4-byte aligned"; return ALBIREO_EINVAL; }
+        a.exp1 = ext->exp1; a.exp1_stride = ext->exp1_stride_elems ? ext->exp1_stride_elems : V;
+    }
+    if (ext->backfill_ids) {
+        if (ext->backfill_len < 1) { *why = "backfill_ids needs backfill_len >= 1"; return ALBIREO_EINVAL; }
+        a.backfill_ids = ext->backfill_ids; a.backfill_index = ext->backfill_index; a.backfill_len = ext->backfill_len;
+    }
+    if (ext->feedback_ring) {
+        if (ext->feedback_cap < 1 || ext->feedback_head < 0) { *why = "feedback_ring needs feedback_cap >= 1 and feedback_head >= 0"; return ALBIREO_EINVAL; }
+        if ((uintptr_t)ext->feedback_ring % 8) { *why = "feedback_ring not 8-byte aligned"; return ALBIREO_EINVAL; }
+        a.feedback_ring = (unsigned long long *)ext->feedback_ring; a.feedback_cap = ext->feedback_cap;
+        a.feedback_head = ext->feedback_head % ext->feedback_cap;
+    }
+    return ALBIREO_OK;
+}
+
+void launch_sample_kernel(int dtype, int B, size_t smem, cudaStream_t st, const SampleArgs &a) {
+    if (dtype == ALBIREO_F32) albireo_sample_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(a);
+    else if (dtype == ALBIREO_BF16) albireo_sample_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(a);
+    else albireo_sample_kernel<ALBIREO_F16><<<B, NT, smem, st>>>(a);
+}
+// Lets every instantiation use the device's opt-in shared memory; gives the dynamic bytes available
+// to a CTA (the opt-in limit less the largest static use), or 0 with *err set.
+size_t enable_large_smem(int device, cudaError_t *err) {
+    int optin = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    cudaFuncAttributes f0, f1, f2;
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&f0, albireo_sample_kernel<ALBIREO_F32>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&f1, albireo_sample_kernel<ALBIREO_BF16>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&f2, albireo_sample_kernel<ALBIREO_F16>);
+    if (e != cudaSuccess) { *err = e; return 0; }
+    size_t st = f0.sharedSizeBytes > f1.sharedSizeBytes ? f0.sharedSizeBytes : f1.sharedSizeBytes;
+    if (f2.sharedSizeBytes > st) st = f2.sharedSizeBytes;
+    if ((size_t)optin <= st) { *err = cudaErrorInvalidValue; return 0; }
+    const size_t smem = (size_t)optin - st;
+    e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    *err = e;
+    return e == cudaSuccess ? smem : 0;
+}
 
 }  // namespace
 
@@ -1751,20 +1879,10 @@ extern "C" int albireo_sample_init(albireo_sampler_t **out, int32_t device, int3
     if (cudaGetDevice(&prev) != cudaSuccess) return ALBIREO_ECUDA;
     if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return ALBIREO_ECUDA; }
     // opt in to the largest dynamic shared memory a CTA may have on this device
-    int optin = 0;
-    cudaError_t e0 = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
-    cudaFuncAttributes fa32, fa16;
-    cudaError_t e1 = cudaFuncGetAttributes(&fa32, albireo_sample_kernel<ALBIREO_F32>);
-    cudaError_t e2 = cudaFuncGetAttributes(&fa16, albireo_sample_kernel<ALBIREO_BF16>);
-    size_t smem = 0;
-    if (e0 == cudaSuccess && e1 == cudaSuccess && e2 == cudaSuccess) {
-        const size_t stat = fa32.sharedSizeBytes > fa16.sharedSizeBytes ? fa32.sharedSizeBytes : fa16.sharedSizeBytes;
-        smem = (size_t)optin > stat ? (size_t)optin - stat : 0;
-        e1 = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        e2 = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    }
+    cudaError_t e0 = cudaSuccess;
+    const size_t smem = enable_large_smem(device, &e0);
     if (prev >= 0 && prev != device) cudaSetDevice(prev);
-    if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); return ALBIREO_ECUDA; }
+    if (e0 != cudaSuccess) { cudaGetLastError(); return ALBIREO_ECUDA; }
     if (smem_bytes_for(max_vocab, true, 2) > smem) return ALBIREO_EUNSUPPORTED;
 
     albireo_sampler *h = new (std::nothrow) albireo_sampler();
@@ -1789,7 +1907,7 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
     if (B == 0) return ALBIREO_OK;
     if (B < 0 || B > h->max_rows) { set_err(h, "B out of range%s", ""); return ALBIREO_EINVAL; }
     if (V < 1 || V > h->max_vocab) { set_err(h, "V out of range%s", ""); return ALBIREO_EINVAL; }
-    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16) { set_err(h, "unknown dtype%s", ""); return ALBIREO_EINVAL; }
+    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16 && dtype != ALBIREO_F16) { set_err(h, "unknown dtype%s", ""); return ALBIREO_EINVAL; }
     if (!logits || !out_tokens || !out_logprobs) { set_err(h, "NULL logits or output%s", ""); return ALBIREO_EINVAL; }
     if ((history_ids == nullptr) != (history_offsets == nullptr)) { set_err(h, "history_ids and history_offsets must both be given%s", ""); return ALBIREO_EINVAL; }
     const size_t esize = dtype == ALBIREO_F32 ? 4 : 2;
@@ -1806,20 +1924,9 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
     a.ws_counts = (uint32_t *)(h->workspace + WS_HEADER);
     a.ws_counts_cap = h->max_history_total;
     if (ext) {
-        if (ext->struct_size != sizeof(albireo_sample_ext_t)) { set_err(h, "ext->struct_size mismatch%s", ""); return ALBIREO_EINVAL; }
-        if (ext->row_stride_elems != 0) {
-            if (ext->row_stride_elems < V) { set_err(h, "row stride smaller than V%s", ""); return ALBIREO_EINVAL; }
-            a.row_stride = ext->row_stride_elems;
-        }
-        a.row_base = ext->row_base; a.flags = ext->flags;
-        if (ext->num_top < 0 || ext->num_top > ALBIREO_MAX_NUM_TOP) { set_err(h, "num_top out of range%s", ""); return ALBIREO_EUNSUPPORTED; }
-        if (ext->num_top > 0 && (!ext->out_top_ids || !ext->out_top_logprobs)) { set_err(h, "num_top > 0 needs both top-N outputs%s", ""); return ALBIREO_EINVAL; }
-        a.num_top = ext->num_top; a.out_top_ids = ext->out_top_ids; a.out_top_logprobs = ext->out_top_logprobs;
-        a.out_num_kept = ext->out_num_kept; a.out_num_topk = ext->out_num_topk;
-        if (ext->dbg_cap < 0 || (ext->dbg_cap > 0 && !ext->dbg_topk_ids)) { set_err(h, "bad dbg_cap / dbg_topk_ids%s", ""); return ALBIREO_EINVAL; }
-        a.dbg_cap = ext->dbg_topk_ids ? ext->dbg_cap : 0;
-        a.dbg_topk_ids = ext->dbg_cap > 0 ? ext->dbg_topk_ids : nullptr;
-        a.out_row_status = ext->out_row_status;
+        const char *why = nullptr;
+        const int rc = apply_ext(a, ext, B, V, &why);
+        if (rc != ALBIREO_OK) { set_err(h, "%s", why); return rc; }
     }
     int cur = -1;
     if (cudaGetDevice(&cur) != cudaSuccess || cur != h->device) { cudaGetLastError(); set_err(h, "the handle's device is not current%s", ""); return ALBIREO_EINVAL; }
@@ -1829,8 +1936,7 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
     while (smem > h->max_smem && a.nstages > 2) smem = smem_bytes_for(V, history_ids != nullptr, --a.nstages);
     if (smem > h->max_smem) { set_err(h, "vocabulary too large for the on-chip tables%s", ""); return ALBIREO_EUNSUPPORTED; }
     cudaStream_t st = (cudaStream_t)stream;
-    if (dtype == ALBIREO_F32) albireo_sample_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(a);
-    else albireo_sample_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(a);
+    launch_sample_kernel(dtype, B, smem, st, a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_err(h, "kernel launch failed: %s", cudaGetErrorString(e)); return ALBIREO_ECUDA; }
     h->launches += 1;
@@ -1848,7 +1954,7 @@ extern "C" int albireo_sample_host(albireo_sampler_t *h, const void *logits, int
     h->err[0] = 0;
     if (B == 0) return ALBIREO_OK;
     if (B < 0 || B > h->max_rows || V < 1 || V > h->max_vocab) { set_err(h, "B or V out of range%s", ""); return ALBIREO_EINVAL; }
-    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16) { set_err(h, "unknown dtype%s", ""); return ALBIREO_EINVAL; }
+    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16 && dtype != ALBIREO_F16) { set_err(h, "unknown dtype%s", ""); return ALBIREO_EINVAL; }
     if (!logits || !out_tokens || !out_logprobs) { set_err(h, "NULL logits or output%s", ""); return ALBIREO_EINVAL; }
     if ((history_ids == nullptr) != (history_offsets == nullptr) || history_total < 0 || history_total > h->max_history_total) {
         set_err(h, "bad history arguments%s", ""); return ALBIREO_EINVAL;
@@ -1856,6 +1962,7 @@ extern "C" int albireo_sample_host(albireo_sampler_t *h, const void *logits, int
     if (ext && ext->struct_size != sizeof(albireo_sample_ext_t)) { set_err(h, "ext->struct_size mismatch%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->row_stride_elems != 0 && ext->row_stride_elems != V) { set_err(h, "host entry needs dense rows%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->dbg_cap > 0) { set_err(h, "host entry has no debug output%s", ""); return ALBIREO_EINVAL; }
+    if (ext && (ext->exp1 || ext->backfill_ids || ext->feedback_ring)) { set_err(h, "host entry takes no exp1 table and no early-feedback targets%s", ""); return ALBIREO_EINVAL; }
     const size_t base = albireo_sample_workspace_bytes(h->max_rows, h->max_vocab, h->max_history_total);
     if (h->workspace_bytes < base + albireo_sample_host_staging_bytes(h->max_rows, h->max_vocab, h->max_history_total)) {
         set_err(h, "workspace given to init has no staging space%s", ""); return ALBIREO_EINVAL;
@@ -1971,18 +2078,7 @@ int fixed_setup(int dev, FixedDeviceState **out) {
         void *ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&ptr, g_fixed_counts);
         if (e != cudaSuccess || !ptr) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e)); }
-        int optin = 0;
-        e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-        cudaFuncAttributes fa32, fa16;
-        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa32, albireo_sample_kernel<ALBIREO_F32>);
-        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa16, albireo_sample_kernel<ALBIREO_BF16>);
-        size_t smem = 0;
-        if (e == cudaSuccess) {
-            const size_t stat = fa32.sharedSizeBytes > fa16.sharedSizeBytes ? fa32.sharedSizeBytes : fa16.sharedSizeBytes;
-            smem = (size_t)optin > stat ? (size_t)optin - stat : 0;
-            e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        }
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const size_t smem = enable_large_smem(dev, &e);
         if (e != cudaSuccess) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "kernel set-up failed: %s", cudaGetErrorString(e)); }
         d.counts = (uint32_t *)ptr; d.max_smem = smem; d.ready = true;
     }
@@ -2004,7 +2100,7 @@ extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32
     if (B < 0) return fixed_fail(ALBIREO_EINVAL, "B is negative%s", "");
     if (V < 1) return fixed_fail(ALBIREO_EINVAL, "V is not positive%s", "");
     if (V > ALBIREO_MAX_VOCAB) return fixed_fail(ALBIREO_EUNSUPPORTED, "V exceeds ALBIREO_MAX_VOCAB%s", "");
-    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16) return fixed_fail(ALBIREO_EINVAL, "unknown dtype%s", "");
+    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16 && dtype != ALBIREO_F16) return fixed_fail(ALBIREO_EINVAL, "unknown dtype%s", "");
     if (!logits || !out_tokens || !out_logprobs) return fixed_fail(ALBIREO_EINVAL, "NULL logits or output%s", "");
     if ((history_ids == nullptr) != (history_offsets == nullptr)) return fixed_fail(ALBIREO_EINVAL, "history_ids and history_offsets must both be given%s", "");
     if (history_total < 0) return fixed_fail(ALBIREO_EINVAL, "history_total is negative%s", "");
@@ -2022,20 +2118,9 @@ extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32
     a.seeds = seeds; a.step = step;
     a.out_tokens = out_tokens; a.out_logprobs = out_logprobs;
     if (ext) {
-        if (ext->struct_size != sizeof(albireo_sample_ext_t)) return fixed_fail(ALBIREO_EINVAL, "ext->struct_size mismatch%s", "");
-        if (ext->row_stride_elems != 0) {
-            if (ext->row_stride_elems < V) return fixed_fail(ALBIREO_EINVAL, "row stride smaller than V%s", "");
-            a.row_stride = ext->row_stride_elems;
-        }
-        a.row_base = ext->row_base; a.flags = ext->flags;
-        if (ext->num_top < 0 || ext->num_top > ALBIREO_MAX_NUM_TOP) return fixed_fail(ALBIREO_EUNSUPPORTED, "num_top out of range%s", "");
-        if (ext->num_top > 0 && (!ext->out_top_ids || !ext->out_top_logprobs)) return fixed_fail(ALBIREO_EINVAL, "num_top > 0 needs both top-N outputs%s", "");
-        a.num_top = ext->num_top; a.out_top_ids = ext->out_top_ids; a.out_top_logprobs = ext->out_top_logprobs;
-        a.out_num_kept = ext->out_num_kept; a.out_num_topk = ext->out_num_topk;
-        if (ext->dbg_cap < 0 || (ext->dbg_cap > 0 && !ext->dbg_topk_ids)) return fixed_fail(ALBIREO_EINVAL, "bad dbg_cap / dbg_topk_ids%s", "");
-        a.dbg_cap = ext->dbg_topk_ids ? ext->dbg_cap : 0;
-        a.dbg_topk_ids = ext->dbg_cap > 0 ? ext->dbg_topk_ids : nullptr;
-        a.out_row_status = ext->out_row_status;
+        const char *why = nullptr;
+        const int rc = apply_ext(a, ext, B, V, &why);
+        if (rc != ALBIREO_OK) return fixed_fail(rc, "%s", why);
     }
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "cudaGetDevice failed%s", ""); }
@@ -2050,8 +2135,7 @@ extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32
     while (smem > d->max_smem && a.nstages > 2) smem = smem_bytes_for(V, history_ids != nullptr, --a.nstages);
     if (smem > d->max_smem) return fixed_fail(ALBIREO_EUNSUPPORTED, "vocabulary too large for the on-chip tables%s", "");
     cudaStream_t st = (cudaStream_t)stream;
-    if (dtype == ALBIREO_F32) albireo_sample_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(a);
-    else albireo_sample_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(a);
+    launch_sample_kernel(dtype, B, smem, st, a);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fixed_fail(ALBIREO_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
     return ALBIREO_OK;

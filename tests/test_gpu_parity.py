@@ -107,6 +107,7 @@ def test_degenerate_rows(binding, sampler, dtype, flags):
     rows.append(np.sort((rng.standard_normal(V) * 3).astype(np.float32))[::-1].copy())   # descending
     r = np.zeros(V, np.float32); r[::2] = -0.0                                 # signed zeros
     rows.append(r)
+    rows.append((rng.standard_normal(V) * 2000).astype(np.float32))            # gaps far wider than the value bins
     x = np.stack(rows)
     n = x.shape[0]
     variants = [

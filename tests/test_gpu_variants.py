@@ -1,0 +1,204 @@
+"""Parity of the sampler's variants with the CPU oracle: binary16 logits (the paper's models are
+FP16, §8.1), pre-generated Exp(1) variates (§6.2) and the early-feedback targets (§5.2)."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import albireo_oracle as O
+from paper_2606_01927_b200 import workloads as W
+
+from parity import EXCUSED_FRACTION, compare, compare_top_lists, to_host
+
+pytestmark = pytest.mark.gpu
+
+DBG_CAP = 128
+_CORES = len(os.sched_getaffinity(0))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2606_01927_b200 import binding as Bd
+    return Bd
+
+
+@pytest.fixture(scope="module")
+def sampler(binding):
+    s = binding.Sampler(max_rows=512, max_vocab=152064 + 64, max_history_total=1 << 21)
+    yield s
+    s.close()
+
+
+def run(binding, sampler, w, *, flags=0, **kw):
+    t = binding.workload_tensors(w, sampler.device)
+    t.pop("backfill_index", None)
+    out = sampler.albireo_sample(t.pop("logits"), **t, row_base=w.row_base, num_top=w.num_top,
+                                 want_counts=True, dbg_cap=DBG_CAP, want_status=True, flags=flags, **kw)
+    torch.cuda.synchronize()
+    return to_host(out)
+
+
+def check(binding, sampler, w, *, flags=0, allow_excused=1):
+    ref = O.sample(w, threads=_CORES, topk_cap=DBG_CAP)
+    g = run(binding, sampler, w, flags=flags)
+    rep = compare(w, g, ref, dbg_cap=DBG_CAP)
+    print(rep.summary())
+    assert rep.ok(), rep.failures[:5]
+    assert len(rep.excused) <= max(allow_excused, math.floor(EXCUSED_FRACTION * w.B)), rep.excused[:5]
+    bad = compare_top_lists(w, g, ref)
+    assert not bad, bad[:3]
+    return g, ref
+
+
+# ------------------------------------------------------------------ binary16 logits
+
+F16_SMALL = [(201, 48, 1000, None), (202, 40, 4099, None), (203, 32, 9001, 0.5), (204, 12, 70001, None), (205, 64, 17, None)]
+
+
+@pytest.mark.parametrize("seed,B,V,q", F16_SMALL)
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_f16_small_mixed_parameters(binding, sampler, seed, B, V, q, flags):
+    w = W.as_f16(W.random_small(seed, B=B, V=V, dtype=W.F32, quantise=q))
+    w.num_top = 5
+    check(binding, sampler, w, flags=flags)
+
+
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_f16_degenerate_rows(binding, sampler, flags):
+    V = 20000
+    rng = np.random.default_rng(23)
+    rows = [np.full(V, 1.5, np.float32)]                                       # all equal
+    r = np.full(V, -np.inf, np.float32); r[[5, 77, 19999]] = [1.0, 1.0, 0.5]  # fewer finite than k
+    rows.append(r)
+    rows.append((rng.standard_normal(V) * 1e-6).astype(np.float32))            # binary16 subnormals and signed zeros
+    r = rng.standard_normal(V).astype(np.float32); r[1234] += 30               # one-hot like
+    rows.append(r)
+    rows.append(np.round(rng.standard_normal(V) * 2).astype(np.float32))       # thousands of ties at the k-th value
+    rows.append((rng.standard_normal(V) * 2000).astype(np.float32))            # near the top of the binary16 range
+    x = np.stack(rows)
+    n = x.shape[0]
+    variants = [
+        dict(temperature=np.full(n, 0.8, np.float32), top_k=np.full(n, 50, np.int32)),
+        dict(temperature=np.full(n, 1.0, np.float32), top_k=np.full(n, 40, np.int32), top_p=np.full(n, 0.9, np.float32)),
+        dict(temperature=np.full(n, 1.0, np.float32), min_p=np.full(n, 0.05, np.float32), top_p=np.full(n, 0.95, np.float32)),
+        dict(temperature=np.full(n, 0.7, np.float32), top_p=np.full(n, 0.5, np.float32)),
+        dict(temperature=np.zeros(n, np.float32)),
+        dict(temperature=np.full(n, 1e-4, np.float32), top_k=np.full(n, 20, np.int32)),   # a very small temperature
+    ]
+    for i, kw in enumerate(variants):
+        w = W.as_f16(W.Workload(f"f16deg{i}", n, V, W.F32, x, seeds=np.arange(n, dtype=np.uint64) + 3, step=9,
+                                num_top=8, **kw))
+        check(binding, sampler, w, flags=flags)
+
+
+def test_f16_full_vocabulary_rows(binding, sampler):
+    w = W.as_f16(W.config2(B=48))
+    g, _ = check(binding, sampler, w)
+    assert (g["row_status"] & 1).sum() == 0            # every row on the single-pass path
+
+
+def test_f16_history_rows(binding, sampler):
+    check(binding, sampler, W.as_f16(W.config3(B=24)))
+
+
+# ------------------------------------------------------------------ pre-generated Exp(1) variates
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_exp1_table_small(binding, sampler, dtype, flags):
+    w = W.with_exp1(W.random_small(301, B=40, V=4099, dtype=dtype), seed=5)
+    w.num_top = 4
+    check(binding, sampler, w, flags=flags)
+
+
+def test_exp1_table_full_vocabulary(binding, sampler):
+    base = W.config4(B=32)
+    g, ref = check(binding, sampler, W.with_exp1(base, seed=6))
+    # the table, not the seeds, decides: the counter-based tokens of the same rows differ somewhere
+    plain = O.sample(base, threads=_CORES)
+    assert (plain.tokens != ref.tokens).any()
+
+
+def test_exp1_forced_winner_and_row_stride(binding, sampler):
+    w = W.with_exp1(W.random_small(302, B=16, V=2000, dtype=W.BF16, with_history=False), seed=8)
+    w.temperature[:] = 1.0
+    w.top_k[:] = 0
+    w.top_p[:] = 1.0
+    w.min_p[:] = 0.0
+    forced = np.arange(16) * 100 + 7
+    w.exp1[np.arange(16), forced] = np.float32(1e-35)       # -ln E = 80: beats any score gap here
+    t = binding.workload_tensors(w, sampler.device)
+    wide = torch.full((16, 2000 + 40), float("nan"), device=sampler.device)
+    wide[:, :2000] = t.pop("exp1")
+    out = sampler.albireo_sample(t.pop("logits"), **t, exp1=wide[:, :2000])
+    torch.cuda.synchronize()
+    assert out.tokens.cpu().tolist() == forced.tolist()
+
+
+# ------------------------------------------------------------------ early feedback
+
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_backfill_and_feedback_ring(binding, sampler, flags):
+    w = W.with_backfill(W.random_small(401, B=50, V=3000, dtype=W.BF16))
+    w.row_base = 1000
+    ref = O.sample(w, threads=_CORES)
+    dev = sampler.device
+    ids_next = torch.full((w.backfill_len,), -7, dtype=torch.int32, device=dev)
+    index = torch.from_numpy(w.backfill_index).to(dev)
+    ring_dev = torch.full((64,), -1, dtype=torch.int64, device=dev)
+    g = run(binding, sampler, w, flags=flags, backfill_ids=ids_next, backfill_index=index,
+            feedback_ring=ring_dev, feedback_head=60)
+    tok = g["tokens"]
+    assert (tok == ref.tokens).all()
+    got = ids_next.cpu().numpy()
+    want = np.full(w.backfill_len, -7, dtype=np.int32)
+    for b in range(w.B):
+        if w.backfill_index[b] >= 0:
+            want[w.backfill_index[b]] = tok[b]
+    assert (got == want).all()
+    ring = ring_dev.cpu().numpy()
+    for b in range(w.B):
+        rec = int(ring[(60 + b) % 64])
+        assert rec >> 32 == 1000 + b and (rec & 0xFFFFFFFF) == tok[b]
+    for slot in set(range(64)) - {(60 + b) % 64 for b in range(w.B)}:
+        assert ring[slot] == -1
+
+
+def test_feedback_ring_in_pinned_host_memory_and_identity_map(binding, sampler):
+    w = W.random_small(402, B=20, V=3000, dtype=W.F32)
+    ref = O.sample(w, threads=_CORES)
+    ring = torch.full((32,), -1, dtype=torch.int64).pin_memory()
+    ids_next = torch.full((w.B,), -7, dtype=torch.int32, device=sampler.device)
+    g = run(binding, sampler, w, backfill_ids=ids_next, feedback_ring=ring)      # no index: row b -> slot b
+    assert (g["tokens"] == ref.tokens).all()
+    assert (ids_next.cpu().numpy() == ref.tokens).all()
+    r = ring.numpy()
+    assert [int(v) & 0xFFFFFFFF for v in r[: w.B]] == ref.tokens.tolist()
+    assert [int(v) >> 32 for v in r[: w.B]] == list(range(w.B))
+    assert (r[w.B:] == -1).all()
+
+
+def test_backfill_index_out_of_range_is_flagged_and_skipped(binding, sampler):
+    w = W.random_small(403, B=8, V=500, dtype=W.F32, with_history=False)
+    ids_next = torch.full((4,), -7, dtype=torch.int32, device=sampler.device)
+    index = torch.tensor([0, 1, 2, 3, 4, 100, -1, -5], dtype=torch.int32, device=sampler.device)
+    g = run(binding, sampler, w, backfill_ids=ids_next, backfill_index=index)
+    assert (ids_next.cpu().numpy() == g["tokens"][:4]).all()
+    assert [(int(s) >> 1) & 1 for s in g["row_status"]] == [0, 0, 0, 0, 1, 1, 0, 0]
+
+
+def test_variant_argument_errors(binding, sampler):
+    w = W.random_small(404, B=4, V=500, dtype=W.F32, with_history=False)
+    t = binding.workload_tensors(w, sampler.device)
+    lg = t.pop("logits")
+    n0 = sampler.launch_count()
+    with pytest.raises(ValueError):
+        sampler.albireo_sample(lg, **t, exp1=torch.ones((4, 500), dtype=torch.float64, device=sampler.device))
+    with pytest.raises(binding.AlbireoError):
+        sampler.albireo_sample(lg, **t, exp1=torch.ones((4, 400), device=sampler.device))   # row stride < V
+    with pytest.raises(binding.AlbireoError):
+        sampler.albireo_sample(lg, **t, feedback_ring=torch.zeros(8, dtype=torch.int64, device=sampler.device),
+                               feedback_head=-1)
+    assert sampler.launch_count() == n0
