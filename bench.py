@@ -163,6 +163,9 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch each step from Python instead of one CUDA graph")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--general-path", action="store_true", help="force every row down the general path")
+    ap.add_argument("--variant", default="none", choices=["none", "f16", "exp1", "feedback"],
+                    help="the same workload as binary16 logits, with a pre-generated Exp(1) table, or with the "
+                         "early-feedback targets (next input ids + pinned host ring)")
     ap.add_argument("--read-ceiling", action="store_true",
                     help="only run the read-ceiling tool (a kernel that just reads the same bytes) and print its table")
     args = ap.parse_args()
@@ -199,6 +202,12 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     w = W.make(args.workload)
+    if args.variant == "f16":
+        w = W.as_f16(w)
+    elif args.variant == "exp1":
+        w = W.with_exp1(w)
+    elif args.variant == "feedback":
+        w = W.with_backfill(w)
     w.row_base = rank * w.B                      # global row ids: draws do not depend on the sharding
     htot = 0 if w.history_ids is None else int(w.history_ids.size)
     sampler = binding.Sampler(max_rows=w.B, max_vocab=w.V, max_history_total=htot, device=dev, host_staging=True)
@@ -210,6 +219,9 @@ def main():
     out_lp = torch.empty(w.B, dtype=torch.float32, device=dev)
     flags = binding.FLAG_FORCE_GENERAL if args.general_path else 0
     stream = torch.cuda.Stream(device=dev)
+    if args.variant == "feedback":
+        t["backfill_ids"] = torch.zeros(w.backfill_len, dtype=torch.int32, device=dev)
+        t["feedback_ring"] = torch.full((2 * w.B,), -1, dtype=torch.int64).pin_memory()
 
     def step(i, st):
         sampler.albireo_sample(bufs[i % N_ROTATING], **t, out_tokens=out_tok, out_logprobs=out_lp, stream=st,
@@ -279,6 +291,7 @@ def main():
     # end to end: host buffers through the C-ABI host entry, copies inside the timed region
     th = binding.workload_tensors(w, "cpu", pinned=True)
     h_logits = th.pop("logits")
+    th.pop("exp1", None); th.pop("backfill_index", None)      # device-only options: the host entry runs the plain call
     h_tok = torch.empty(w.B, dtype=torch.int32, pin_memory=True)
     h_lp = torch.empty(w.B, dtype=torch.float32, pin_memory=True)
     h2d = sum(int(v.numel() * v.element_size()) for v in [h_logits] + [x for x in th.values() if torch.is_tensor(x)])
@@ -314,6 +327,7 @@ def main():
                 "l2": f"{N_ROTATING} rotating logits buffers ({N_ROTATING * w.logit_bytes / 1e6:.0f} MB per GPU) so no call finds its rows in the 126 MB L2",
                 "launch": "one CUDA graph of K launches" if graph is not None else "K launches from the host",
                 "path": "general path forced" if args.general_path else "automatic",
+                "variant": args.variant,
             },
             "tokens_per_s": value,
             "roofline": {
