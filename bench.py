@@ -151,6 +151,71 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def run_sequence_parallel(args, rank, world, local_rank):
+    """Secondary mode (section 6.1): the batch's logits start as vocabulary shards [s, v/t], one per
+    rank; a step is all-to-all + sample local rows + gather of the tokens ("a2a"), or the gather-to-one
+    arrangement it replaces ("gather").  Total work is fixed as N grows (strong scaling)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2606_01927_b200 import _build
+    _build.build()
+    from paper_2606_01927_b200 import binding, sequence_parallel as SP, workloads as W
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if not dist.is_initialized():
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29571")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    w = W.make(args.workload)
+    s_rows, V = w.B, w.V
+    if V % world or (V // world * w.elem_size) % 16:
+        raise SystemExit("the vocabulary does not split into 16-byte aligned shards over this many ranks")
+    vs = V // world
+    t_full = binding.workload_tensors(w, dev)
+    full = t_full.pop("logits")
+    shards = [full[:, rank * vs:(rank + 1) * vs].contiguous()]
+    shards += [torch.roll(shards[0], shifts=i, dims=0).contiguous() for i in range(1, N_ROTATING)]
+    del full
+    lay = SP.layout(s_rows)
+    htot = 0 if w.history_ids is None else int(w.history_ids.size)
+    sampler = binding.Sampler(max_rows=s_rows, max_vocab=V, max_history_total=htot, device=dev)
+    meta_all = {k: v for k, v in t_full.items() if k != "step"}
+    meta_local = SP.scatter_metadata(meta_all if rank == 0 else None, lay, dev)
+    fn = SP.cuda_sample_fn(sampler)
+    recv = torch.empty((world, lay.rows, vs), dtype=shards[0].dtype, device=dev)
+
+    def step(i):
+        if args.sequence_parallel == "a2a":
+            return SP.sample_step(fn, shards[i % N_ROTATING], meta_local, lay, step=w.step, recv=recv)
+        return SP.gather_then_sample_step(fn, shards[i % N_ROTATING], meta_all, s_rows, step=w.step)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize(dev)
+    dist.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    dist.barrier()
+    tt = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ms = float(tt.item()) / args.steps
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": s_rows / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w), "mode": "sequence-parallel " + args.sequence_parallel,
+                       "rows_per_gpu": lay.rows, "launch": "K steps from the host (collectives + one kernel each)"},
+            "gpu_launches": sampler.launch_count() - args.warmup}))
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -166,6 +231,9 @@ def main():
     ap.add_argument("--variant", default="none", choices=["none", "f16", "exp1", "feedback"],
                     help="the same workload as binary16 logits, with a pre-generated Exp(1) table, or with the "
                          "early-feedback targets (next input ids + pinned host ring)")
+    ap.add_argument("--sequence-parallel", default=None, choices=["a2a", "gather"],
+                    help="secondary mode: logits start as per-rank vocabulary shards; time all-to-all + sample + "
+                         "gather (a2a) or the gather-to-one-rank arrangement it replaces (gather)")
     ap.add_argument("--read-ceiling", action="store_true",
                     help="only run the read-ceiling tool (a kernel that just reads the same bytes) and print its table")
     args = ap.parse_args()
@@ -180,6 +248,9 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             run_reference(args, W.make(args.workload))
+        return
+    if args.sequence_parallel:
+        run_sequence_parallel(args, rank, world, local_rank)
         return
     if args.read_ceiling:
         if rank == 0:

@@ -112,6 +112,18 @@ typedef struct albireo_sample_ext {
     uint64_t *feedback_ring;       /* [feedback_cap] device-visible, 8-byte aligned, or NULL */
     int64_t feedback_cap;
     int64_t feedback_head;
+
+    /* Rows in pieces (sequence-parallel sampling, section 6.1 steps 2-3): after the all-to-all
+       that turns vocabulary shards into row shards, a worker holds each of its rows as
+       num_segments pieces of V / num_segments logits, one per sending worker.  With
+       num_segments >= 2 the sampler reads them where they landed: element i of row b is
+       logits[(i / Vs) * segment_stride_elems + b * row_stride + (i % Vs)], Vs = V / num_segments
+       (row_stride_elems 0 then means Vs).  For the receive buffer [t, B, V/t] of an all-to-all
+       that is segment_stride_elems = B * V / t.  num_segments must divide V and be <= 64; the
+       base pointer and, in bytes, Vs, the row stride and the segment stride must be multiples
+       of 16 (ALBIREO_EUNSUPPORTED otherwise).  0 or 1: rows are contiguous.                */
+    int32_t num_segments;
+    int64_t segment_stride_elems;
 } albireo_sample_ext_t;
 
 /*

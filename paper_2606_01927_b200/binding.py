@@ -50,6 +50,7 @@ class SampleExt(C.Structure):
         ("exp1", C.c_void_p), ("exp1_stride_elems", C.c_int64),
         ("backfill_ids", C.c_void_p), ("backfill_index", C.c_void_p), ("backfill_len", C.c_int64),
         ("feedback_ring", C.c_void_p), ("feedback_cap", C.c_int64), ("feedback_head", C.c_int64),
+        ("num_segments", C.c_int32), ("segment_stride_elems", C.c_int64),
     ]
 
 
@@ -208,10 +209,19 @@ class Sampler:
         ``exp1`` (float32 ``[B, V]``) replaces the counter-based draw by pre-generated Exp(1)
         variates; ``backfill_ids`` / ``backfill_index`` (int32) and ``feedback_ring`` (int64,
         device or pinned host memory) are the early-feedback targets."""
-        if logits.dim() != 2 or logits.stride(1) != 1:
+        nseg = 0
+        if logits.dim() == 3:
+            # rows in pieces, [t, B, V / t]: the receive buffer of the sequence-parallel all-to-all
+            if logits.stride(2) != 1:
+                raise ValueError("logits in pieces must be [t, B, V/t] with unit stride along the last axis")
+            nseg = logits.shape[0]
+            B = logits.shape[1] if B is None else B
+            V = nseg * logits.shape[2] if V is None else V
+        elif logits.dim() != 2 or logits.stride(1) != 1:
             raise ValueError("logits must be [B, V] with unit stride along V")
-        B = logits.shape[0] if B is None else B
-        V = logits.shape[1] if V is None else V
+        else:
+            B = logits.shape[0] if B is None else B
+            V = logits.shape[1] if V is None else V
         dt = _dtype_code(logits)
         dev = logits.device
         if out_tokens is None:
@@ -219,9 +229,15 @@ class Sampler:
         if out_logprobs is None:
             out_logprobs = torch.empty(B, dtype=torch.float32, device=dev)
         row_stride = logits.stride(0) if B > 1 else V
+        if nseg:
+            row_stride = logits.stride(1)
         ext, extra = self._ext(B, "cuda", dev, row_base=row_base, row_stride=0 if row_stride == V else row_stride,
                                num_top=num_top, want_counts=want_counts, dbg_cap=dbg_cap,
                                want_status=want_status, flags=flags)
+        if nseg:
+            ext.num_segments = nseg
+            ext.segment_stride_elems = logits.stride(0)
+            ext.row_stride_elems = row_stride
         if exp1 is not None:
             if exp1.dtype != torch.float32 or exp1.dim() != 2 or exp1.stride(1) != 1 or exp1.device != dev:
                 raise ValueError("exp1 must be a float32 [B, V] tensor on the logits' device")

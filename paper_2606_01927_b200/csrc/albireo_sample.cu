@@ -55,6 +55,8 @@ struct SampleArgs {
     const void *logits;
     int32_t B, V;
     int64_t row_stride;
+    int32_t nseg;               // pieces per row (1: rows are contiguous)
+    int64_t seg_stride;         // elements between consecutive pieces of a row
     const float *temperature;
     const int32_t *top_k;
     const float *top_p, *min_p, *rep, *pres, *freq;
@@ -72,6 +74,7 @@ struct SampleArgs {
     int32_t dbg_cap;
     int32_t *dbg_topk_ids;
     uint32_t *out_row_status;
+    int32_t elem_size;          // host side only: bytes per logit
     int32_t nstages;            // ring depth chosen by the host for this launch
     const float *exp1;          // pre-generated Exp(1) variates [B, exp1_stride], or null: counter-based draw
     int64_t exp1_stride;
@@ -234,6 +237,10 @@ __device__ u64 block_exscan_u64(BlockScratch &s, u64 v, u64 &total) {
 struct RowCtx {
     const void *row;       // first logit of the row
     int V;
+    // a row may arrive as nseg equal pieces of Vs elements (vocabulary shards as the all-to-all of
+    // sequence-parallel sampling leaves them, section 6.1 step 2), seg_bytes apart; nseg == 1: one piece
+    int nseg, Vs;
+    int64_t seg_bytes;
     float invT, r, p, f;
     bool has_hist;
     const uint32_t *bitmap;   // V bits (+1 pad word): token appears in the history
@@ -299,6 +306,23 @@ template <> struct Elem<ALBIREO_F16> {
     }
 };
 
+// address of element i of the row
+template <int DT>
+__device__ __forceinline__ const void *elem_ptr(const RowCtx &c, int i) {
+    if (c.nseg == 1) return (const char *)c.row + (size_t)i * Elem<DT>::SIZE;
+    const int j = i / c.Vs;
+    return (const char *)c.row + (size_t)j * (size_t)c.seg_bytes + (size_t)(i - j * c.Vs) * Elem<DT>::SIZE;
+}
+// address of the row's v-th 16-byte vector (rows in pieces are 16-byte aligned piece by piece, so
+// their vectors start at element 0 and none straddles two pieces)
+template <int DT>
+__device__ __forceinline__ const uint4 *vec_ptr(const RowCtx &c, const uint4 *vp, int v) {
+    if (c.nseg == 1) return vp + v;
+    const int vps = c.Vs / Elem<DT>::PER_VEC;
+    const int j = v / vps;
+    return (const uint4 *)((const char *)c.row + (size_t)j * (size_t)c.seg_bytes) + (v - j * vps);
+}
+
 __device__ __forceinline__ float score_of(const RowCtx &c, int i, float x) {
     float a = x;
     if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) a = penalise(c, i, x);
@@ -322,8 +346,8 @@ __device__ __forceinline__ void for_each_score(const RowCtx &c, F &&fn) {
     const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
     for (int v0 = threadIdx.x; v0 < nvec; v0 += 2 * NT) {
         const int v1 = v0 + NT;
-        const uint4 q0 = __ldg(vp + v0);
-        const uint4 q1 = v1 < nvec ? __ldg(vp + v1) : q0;
+        const uint4 q0 = __ldg(vec_ptr<DT>(c, vp, v0));
+        const uint4 q1 = v1 < nvec ? __ldg(vec_ptr<DT>(c, vp, v1)) : q0;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             if (u == 1 && v1 >= nvec) break;
@@ -340,12 +364,12 @@ __device__ __forceinline__ void for_each_score(const RowCtx &c, F &&fn) {
     for (int q = threadIdx.x; q < head + (V - tail0); q += NT) {
         const int i = q < head ? q : tail0 + (q - head);
         if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
-        fn(i, __fmul_rn(E::load(c.row, i), c.invT));
+        fn(i, __fmul_rn(E::load(elem_ptr<DT>(c, i), 0), c.invT));
     }
     if (c.has_hist) {
         for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
             const int i = hist_id_of_rank(c, r);
-            const float x = E::load(c.row, i);
+            const float x = E::load(elem_ptr<DT>(c, i), 0);
             float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
             av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(c.counts[r])));
             av = __fsub_rn(av, c.p);
@@ -800,7 +824,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const u64 G = block_max_u64(s, g_best);
     const int tok = comp_idx(G);
     const double lnS = log((double)S_fx) - LN2_40;
-    float z_tok = score_of(c, tok, Elem<DT>::load(c.row, tok));
+    float z_tok = score_of(c, tok, Elem<DT>::load(elem_ptr<DT>(c, tok), 0));
     out.token = tok;                                   // (a single kept element wins its own race)
     out.logprob = (n_keep == 1) ? 0.0f : (float)(((double)z_tok - (double)zmax) - lnS);
     out.n_keep = (int32_t)n_keep;
@@ -841,6 +865,10 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
 // its copies and leaves.
 
 struct Ring {
+    // source of the copies: vectors per piece of the row and the distance between pieces (a row in
+    // one piece: vps covers the whole row)
+    int vps;
+    int64_t seg_vecs;
     unsigned char *buf;     // nstages * STAGE_BYTES, 128-byte aligned
     uint64_t *bar;          // one mbarrier per stage
     int nstages;
@@ -868,12 +896,22 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+// copies vectors [v0, v0 + nv) of the row to dst, piece by piece; the bytes were announced to `bar`
+__device__ __forceinline__ void ring_copy(const Ring &rg, void *dst, const uint4 *vp, int v0, int nv, uint64_t *bar) {
+    unsigned char *d = (unsigned char *)dst;
+    int j = v0 / rg.vps, off = v0 - j * rg.vps;
+    while (nv > 0) {
+        const int n1 = nv < rg.vps - off ? nv : rg.vps - off;
+        bulk_g2s(d, vp + (int64_t)j * rg.seg_vecs + off, (uint32_t)n1 * 16u, bar);
+        d += (size_t)n1 * 16; nv -= n1; ++j; off = 0;
+    }
+}
 // issues the copy of tile t (called by one thread)
 __device__ __forceinline__ void ring_issue(const Ring &rg, const uint4 *vp, int nvec, int t, int st) {
     const int v0 = t * (NT * TILE_VECS);
     int nv = nvec - v0; if (nv > NT * TILE_VECS) nv = NT * TILE_VECS;
     mbar_expect_tx(&rg.bar[st], (uint32_t)nv * 16u);
-    bulk_g2s(rg.buf + (size_t)st * STAGE_BYTES, vp + v0, (uint32_t)nv * 16u, &rg.bar[st]);
+    ring_copy(rg, rg.buf + (size_t)st * STAGE_BYTES, vp, v0, nv, &rg.bar[st]);
 }
 // Tile 0 arrives in two copies: its first NT vectors (the warm-up slice, one vector per thread) on
 // their own mbarrier so that the threshold can be set up while the rest is still in flight.
@@ -881,10 +919,10 @@ __device__ __forceinline__ void ring_issue_first(const Ring &rg, const uint4 *vp
     const int na = nvec < NT ? nvec : NT;
     int nb = nvec - na; if (nb > NT * (TILE_VECS - 1)) nb = NT * (TILE_VECS - 1);
     mbar_expect_tx(&rg.bar[MAX_STAGES - 1], (uint32_t)na * 16u);
-    bulk_g2s(rg.buf, vp, (uint32_t)na * 16u, &rg.bar[MAX_STAGES - 1]);
+    ring_copy(rg, rg.buf, vp, 0, na, &rg.bar[MAX_STAGES - 1]);
     if (nb > 0) {
         mbar_expect_tx(&rg.bar[0], (uint32_t)nb * 16u);
-        bulk_g2s(rg.buf + (size_t)na * 16, vp + na, (uint32_t)nb * 16u, &rg.bar[0]);
+        ring_copy(rg, rg.buf + (size_t)na * 16, vp, na, nb, &rg.bar[0]);
     } else {
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rg.bar[0])) : "memory");
     }
@@ -1574,7 +1612,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         for (int q = threadIdx.x; q < nscal; q += NT) {
             int i = q < head ? q : tail0 + (q - head);
             if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
-            uint32_t key = key_of(__fmul_rn(E::load(c.row, i), c.invT));
+            uint32_t key = key_of(__fmul_rn(E::load(elem_ptr<DT>(c, i), 0), c.invT));
             if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
         }
     }
@@ -1583,7 +1621,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     if (c.has_hist) {
         for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
             const int i = hist_id_of_rank(c, r);
-            const float x = E::load(c.row, i);
+            const float x = E::load(elem_ptr<DT>(c, i), 0);
             const uint32_t cntv = c.counts[r];
             float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
             av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cntv)));
@@ -1646,6 +1684,8 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     h.acc = h.list + GL_CAP;
     Ring rg;
     rg.nstages = a.nstages;
+    rg.vps = a.nseg > 1 ? (V / a.nseg) / Elem<DT>::PER_VEC : 0x7FFFFFFF;
+    rg.seg_vecs = a.seg_stride * Elem<DT>::SIZE / 16;
     rg.buf = smem + COMMON_BYTES;
     rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
     HistSmem hs;
@@ -1657,6 +1697,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     RowCtx c;
     c.row = (const char *)a.logits + (size_t)b * (size_t)a.row_stride * Elem<DT>::SIZE;
     c.V = V;
+    c.nseg = a.nseg; c.Vs = V / a.nseg; c.seg_bytes = a.seg_stride * Elem<DT>::SIZE;
     // The ring is started before anything else is read, the row's own parameters included: their
     // loads and the first tiles then travel together.  A row that turns out to need the general
     // path waits for these copies before it reuses the shared memory.
@@ -1771,7 +1812,7 @@ int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, cons
     (void)B;
     if (ext->struct_size != sizeof(albireo_sample_ext_t)) { *why = "ext->struct_size mismatch"; return ALBIREO_EINVAL; }
     if (ext->row_stride_elems != 0) {
-        if (ext->row_stride_elems < V) { *why = "row stride smaller than V"; return ALBIREO_EINVAL; }
+        if (ext->row_stride_elems < V && ext->num_segments <= 1) { *why = "row stride smaller than V"; return ALBIREO_EINVAL; }
         a.row_stride = ext->row_stride_elems;
     }
     a.row_base = ext->row_base; a.flags = ext->flags;
@@ -1783,6 +1824,19 @@ int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, cons
     a.dbg_cap = ext->dbg_topk_ids ? ext->dbg_cap : 0;
     a.dbg_topk_ids = ext->dbg_cap > 0 ? ext->dbg_topk_ids : nullptr;
     a.out_row_status = ext->out_row_status;
+    if (ext->num_segments > 1) {
+        // rows in pieces: every piece must start and end on a 16-byte boundary
+        const int64_t esz = a.elem_size, t = ext->num_segments;
+        if (t > 64 || V % t) { *why = "num_segments must divide V and be at most 64"; return ALBIREO_EINVAL; }
+        const int64_t Vs = V / t;
+        if (ext->segment_stride_elems < Vs) { *why = "segment stride smaller than a piece"; return ALBIREO_EINVAL; }
+        if (ext->row_stride_elems == 0) a.row_stride = Vs;
+        if (a.row_stride < Vs) { *why = "row stride smaller than a piece"; return ALBIREO_EINVAL; }
+        if ((Vs * esz) % 16 || (a.row_stride * esz) % 16 || (ext->segment_stride_elems * esz) % 16 || (uintptr_t)a.logits % 16) {
+            *why = "rows in pieces need 16-byte aligned pieces, row stride, segment stride and base"; return ALBIREO_EUNSUPPORTED;
+        }
+        a.nseg = (int32_t)t; a.seg_stride = ext->segment_stride_elems;
+    } else if (ext->num_segments < 0) { *why = "num_segments is negative"; return ALBIREO_EINVAL; }
     if (ext->exp1) {
         if (ext->exp1_stride_elems != 0 && ext->exp1_stride_elems < V) { *why = "exp1 row stride smaller than V"; return ALBIREO_EINVAL; }
         if ((uintptr_t)ext->exp1 % 4) { *why = "exp1 not 4-byte aligned"; return ALBIREO_EINVAL; }
@@ -1915,7 +1969,7 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
 
     SampleArgs a;
     memset(&a, 0, sizeof a);
-    a.logits = logits; a.B = B; a.V = V; a.row_stride = V;
+    a.logits = logits; a.B = B; a.V = V; a.row_stride = V; a.nseg = 1; a.elem_size = (int32_t)esize;
     a.temperature = temperature; a.top_k = top_k; a.top_p = top_p; a.min_p = min_p;
     a.rep = repetition_penalty; a.pres = presence_penalty; a.freq = frequency_penalty;
     a.hist_ids = history_ids; a.hist_off = history_offsets;
@@ -1962,7 +2016,7 @@ extern "C" int albireo_sample_host(albireo_sampler_t *h, const void *logits, int
     if (ext && ext->struct_size != sizeof(albireo_sample_ext_t)) { set_err(h, "ext->struct_size mismatch%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->row_stride_elems != 0 && ext->row_stride_elems != V) { set_err(h, "host entry needs dense rows%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->dbg_cap > 0) { set_err(h, "host entry has no debug output%s", ""); return ALBIREO_EINVAL; }
-    if (ext && (ext->exp1 || ext->backfill_ids || ext->feedback_ring)) { set_err(h, "host entry takes no exp1 table and no early-feedback targets%s", ""); return ALBIREO_EINVAL; }
+    if (ext && (ext->exp1 || ext->backfill_ids || ext->feedback_ring || ext->num_segments > 1)) { set_err(h, "host entry takes no exp1 table, no early-feedback targets and no rows in pieces%s", ""); return ALBIREO_EINVAL; }
     const size_t base = albireo_sample_workspace_bytes(h->max_rows, h->max_vocab, h->max_history_total);
     if (h->workspace_bytes < base + albireo_sample_host_staging_bytes(h->max_rows, h->max_vocab, h->max_history_total)) {
         set_err(h, "workspace given to init has no staging space%s", ""); return ALBIREO_EINVAL;
@@ -2111,7 +2165,7 @@ extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32
 
     SampleArgs a;
     memset(&a, 0, sizeof a);
-    a.logits = logits; a.B = B; a.V = V; a.row_stride = V;
+    a.logits = logits; a.B = B; a.V = V; a.row_stride = V; a.nseg = 1; a.elem_size = (int32_t)esize;
     a.temperature = temperature; a.top_k = top_k; a.top_p = top_p; a.min_p = min_p;
     a.rep = repetition_penalty; a.pres = presence_penalty; a.freq = frequency_penalty;
     a.hist_ids = history_ids; a.hist_off = history_offsets;

@@ -202,3 +202,75 @@ def test_variant_argument_errors(binding, sampler):
         sampler.albireo_sample(lg, **t, feedback_ring=torch.zeros(8, dtype=torch.int64, device=sampler.device),
                                feedback_head=-1)
     assert sampler.launch_count() == n0
+
+
+# ------------------------------------------------------------------ rows in pieces (sequence-parallel layout)
+
+def pieces(logits_2d: torch.Tensor, t: int, pad_rows: int = 0, pad_cols: int = 0) -> torch.Tensor:
+    """[B, V] -> the [t, B, V/t] layout an all-to-all of vocabulary shards leaves (optionally inside a
+    larger allocation so that the strides are not the dense ones)."""
+    B, V = logits_2d.shape
+    Vs = V // t
+    big = torch.zeros((t, B + pad_rows, Vs + pad_cols), dtype=logits_2d.dtype, device=logits_2d.device)
+    for j in range(t):
+        big[j, :B, :Vs] = logits_2d[:, j * Vs:(j + 1) * Vs]
+    return big[:, :B, :Vs]
+
+
+@pytest.mark.parametrize("t,dtype,V,pad", [(2, W.BF16, 8192, (0, 0)), (4, W.BF16, 152064, (0, 0)), (4, W.F32, 40000, (3, 8)),
+                                           (8, W.BF16, 70016, (1, 16)), (4, W.F16, 152064, (0, 0))])
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_rows_in_pieces_match_contiguous_rows(binding, sampler, t, dtype, V, pad, flags):
+    base = W.random_small(500 + t, B=24, V=V, dtype=W.F32 if dtype == W.F16 else dtype)
+    w = W.as_f16(base) if dtype == W.F16 else base
+    w.num_top = 3
+    ref = O.sample(w, threads=_CORES, topk_cap=DBG_CAP)
+    tt = binding.workload_tensors(w, sampler.device)
+    lg = pieces(tt.pop("logits"), t, *pad)
+    out = sampler.albireo_sample(lg, **tt, num_top=w.num_top, want_counts=True, dbg_cap=DBG_CAP, want_status=True, flags=flags)
+    torch.cuda.synchronize()
+    g = to_host(out)
+    rep = compare(w, g, ref, dbg_cap=DBG_CAP)
+    print(rep.summary())
+    assert rep.ok(), rep.failures[:5]
+    assert len(rep.excused) <= 1
+    assert not compare_top_lists(w, g, ref)
+
+
+def test_rows_in_pieces_argument_errors(binding, sampler):
+    w = W.random_small(510, B=4, V=4096, dtype=W.BF16, with_history=False)
+    tt = binding.workload_tensors(w, sampler.device)
+    lg2 = tt.pop("logits")
+    n0 = sampler.launch_count()
+    with pytest.raises(binding.AlbireoError):                   # pieces of 4096 / 3 elements: V not divisible
+        sampler.albireo_sample(pieces(lg2[:, :4095], 3), **tt, V=4096)
+    with pytest.raises(binding.AlbireoError):                   # pieces whose byte length is not a multiple of 16
+        sampler.albireo_sample(pieces(lg2[:, :4088], 2, 0, 4), **tt)
+    assert sampler.launch_count() == n0
+
+
+def test_sequence_parallel_step_on_one_rank(binding, sampler):
+    """The whole sequence-parallel step (all-to-all, sample, gather) through NCCL with a group of one:
+    the collectives are trivial, the code path and the sampler's reading of the pieces are the real ones."""
+    import socket
+    import torch.distributed as dist
+    from paper_2606_01927_b200 import sequence_parallel as SP
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=sampler.device)
+    try:
+        w = W.config4(B=40)
+        ref = O.sample(w, threads=_CORES)
+        tt = binding.workload_tensors(w, sampler.device)
+        shard = tt.pop("logits")
+        step = tt.pop("step")
+        lay = SP.layout(w.B)
+        meta = SP.scatter_metadata(tt, lay, sampler.device)
+        tok, lp = SP.sample_step(SP.cuda_sample_fn(sampler), shard, meta, lay, step=step)
+        torch.cuda.synchronize()
+        assert (tok.cpu().numpy() == ref.tokens).mean() >= 0.97          # cut-boundary rows are judged in the parity tests
+        assert np.abs(lp.cpu().numpy()[tok.cpu().numpy() == ref.tokens] - ref.logprobs[tok.cpu().numpy() == ref.tokens]).max() < 1e-4
+    finally:
+        dist.destroy_process_group()
