@@ -331,6 +331,149 @@ __device__ __forceinline__ float score_of(const RowCtx &c, int i, float x) {
 
 __device__ int hist_id_of_rank(const RowCtx &c, uint32_t r);
 
+// Vector pre-test per dtype, in the domain the test runs in.
+// 16-bit types: raw logits; the threshold is the smallest raw value whose score has key >= tau
+// (packed twice).  x -> fl32(x * invT) is increasing, strictly so on distinct 16-bit values unless
+// the product leaves the fp32 range, so a compare of raw values is a superset of the key test.
+// fp32: scores; the threshold is unkey(tau).
+struct Bf16Packed {
+    typedef __nv_bfloat162 H2;
+    static constexpr uint32_t LO = 0x0080u, HI = 0xFF7Fu, NEG_INF = 0xFF80u;    // order codes of the finite range; -inf pattern
+    static __device__ __forceinline__ float widen(uint32_t bits) { return __uint_as_float(bits << 16); }
+    static __device__ __forceinline__ uint32_t truncate(float x) { return __float_as_uint(x) >> 16; }
+};
+struct F16Packed {
+    typedef __half2 H2;
+    static constexpr uint32_t LO = 0x0400u, HI = 0xFBFFu, NEG_INF = 0xFC00u;
+    static __device__ __forceinline__ float widen(uint32_t bits) { return __half2float(__ushort_as_half((unsigned short)bits)); }
+    static __device__ __forceinline__ uint32_t truncate(float x) { return __half_as_ushort(__float2half_rz(x)); }
+};
+template <int DT> struct VecTest;
+template <class P> struct VecTest16 {
+    typedef typename P::H2 H2;
+    static __device__ uint32_t raw_threshold(uint32_t tau_key, float invT) {
+        // order code of a 16-bit pattern (the analogue of the score key) and back
+        auto bits_of = [](uint32_t kk) { return (kk & 0x8000u) ? (kk & 0x7FFFu) : (~kk & 0xFFFFu); };
+        auto passes = [&](uint32_t kk) {
+            float x = P::widen(bits_of(kk));
+            return key_of(__fmul_rn(x, invT)) >= tau_key;
+        };
+        constexpr uint32_t LO = P::LO, HI = P::HI;             // the finite codes
+        // a guess from an approximate quotient, truncated to 16 bits: the answer is the guess or a
+        // neighbour, so the four codes around it are tried at once instead of one after another
+        const float xg = __fdividef(unkey(tau_key), invT);
+        const uint32_t b16 = P::truncate(xg) & 0xFFFFu;
+        uint32_t k16 = (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
+        k16 = k16 < LO + 2u ? LO + 2u : (k16 > HI - 1u ? HI - 1u : k16);
+        const bool p0 = passes(k16 - 2u), p1 = passes(k16 - 1u), p2 = passes(k16), p3 = passes(k16 + 1u);
+        uint32_t ans = 0;
+        if (p1 && !p0) ans = k16 - 1u;
+        else if (p2 && !p1) ans = k16;
+        else if (p3 && !p2) ans = k16 + 1u;
+        if (ans == 0) {
+            // not bracketed (an extreme temperature, or the ends of the range): a short walk
+            int it = 0;
+            while (it < 16 && k16 > LO && passes(k16)) { --k16; ++it; }
+            while (it < 32 && k16 < HI && !passes(k16)) { ++k16; ++it; }
+            const bool ok = passes(k16) && (k16 == LO || !passes(k16 - 1u));
+            ans = ok ? k16 : 0u;
+        }
+        const uint32_t b = ans ? bits_of(ans) : P::NEG_INF;    // not settled: let everything through
+        return b | (b << 16);
+    }
+    static __device__ __forceinline__ H2 vmax(const uint4 &q) {
+        H2 a = __hmax2(*reinterpret_cast<const H2 *>(&q.x), *reinterpret_cast<const H2 *>(&q.y));
+        H2 b2 = __hmax2(*reinterpret_cast<const H2 *>(&q.z), *reinterpret_cast<const H2 *>(&q.w));
+        return __hmax2(a, b2);
+    }
+    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
+        return __hge2_mask(vmax(q), *reinterpret_cast<const H2 *>(&thr)) != 0u;
+    }
+    static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float) {
+        H2 m = vmax(q[0]);
+#pragma unroll
+        for (int u = 1; u < TILE_VECS; ++u) m = __hmax2(m, vmax(q[u]));
+        return __hge2_mask(m, *reinterpret_cast<const H2 *>(&thr)) != 0u;
+    }
+    // bit e set: raw element e >= the raw threshold (a superset of "score key >= tau")
+    static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float) {
+        const H2 t2 = *reinterpret_cast<const H2 *>(&thr);
+        const uint32_t r0 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.x), t2);
+        const uint32_t r1 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.y), t2);
+        const uint32_t r2 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.z), t2);
+        const uint32_t r3 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.w), t2);
+        return ((r0 & 1u) | ((r0 >> 15) & 2u)) | (((r1 & 1u) | ((r1 >> 15) & 2u)) << 2) |
+               (((r2 & 1u) | ((r2 >> 15) & 2u)) << 4) | (((r3 & 1u) | ((r3 >> 15) & 2u)) << 6);
+    }
+    // key of the score of the vector's largest element (an element of the row)
+    static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) {
+        H2 m = vmax(q);
+        return key_of(__fmul_rn(fmaxf(__low2float(m), __high2float(m)), invT));
+    }
+    static __device__ __forceinline__ uint4 fill() { const uint32_t f = P::NEG_INF | (P::NEG_INF << 16); return make_uint4(f, f, f, f); }
+    // how many of the vector's elements are -inf
+    static __device__ __forceinline__ uint32_t count_neginf(const uint4 &q) {
+        const uint32_t f = P::NEG_INF | (P::NEG_INF << 16);
+        const H2 ninf = *reinterpret_cast<const H2 *>(&f);
+        const uint32_t r0 = __heq2_mask(*reinterpret_cast<const H2 *>(&q.x), ninf), r1 = __heq2_mask(*reinterpret_cast<const H2 *>(&q.y), ninf);
+        const uint32_t r2 = __heq2_mask(*reinterpret_cast<const H2 *>(&q.z), ninf), r3 = __heq2_mask(*reinterpret_cast<const H2 *>(&q.w), ninf);
+        if (!(r0 | r1 | r2 | r3)) return 0u;
+        return (uint32_t)(__popc(r0) + __popc(r1) + __popc(r2) + __popc(r3)) >> 4;
+    }
+};
+template <> struct VecTest<ALBIREO_BF16> : VecTest16<Bf16Packed> {};
+template <> struct VecTest<ALBIREO_F16> : VecTest16<F16Packed> {};
+template <> struct VecTest<ALBIREO_F32> {
+    static __device__ uint32_t raw_threshold(uint32_t tau_key, float) { return __float_as_uint(unkey(tau_key)); }
+    static __device__ __forceinline__ float vmaxz(const uint4 &q, float invT) {
+        return fmaxf(fmaxf(__fmul_rn(__uint_as_float(q.x), invT), __fmul_rn(__uint_as_float(q.y), invT)),
+                     fmaxf(__fmul_rn(__uint_as_float(q.z), invT), __fmul_rn(__uint_as_float(q.w), invT)));
+    }
+    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float invT) {
+        return vmaxz(q, invT) >= __uint_as_float(thr);
+    }
+    static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float invT) {
+        float m = vmaxz(q[0], invT);
+#pragma unroll
+        for (int u = 1; u < TILE_VECS; ++u) m = fmaxf(m, vmaxz(q[u], invT));
+        return m >= __uint_as_float(thr);
+    }
+    static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float invT) {
+        const float t = __uint_as_float(thr);
+        return (uint32_t)(__fmul_rn(__uint_as_float(q.x), invT) >= t) | ((uint32_t)(__fmul_rn(__uint_as_float(q.y), invT) >= t) << 1) |
+               ((uint32_t)(__fmul_rn(__uint_as_float(q.z), invT) >= t) << 2) | ((uint32_t)(__fmul_rn(__uint_as_float(q.w), invT) >= t) << 3);
+    }
+    static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) { return key_of(vmaxz(q, invT)); }
+    static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
+    static __device__ __forceinline__ uint32_t count_neginf(const uint4 &q) {
+        return (uint32_t)(q.x == 0xFF800000u) + (uint32_t)(q.y == 0xFF800000u) + (uint32_t)(q.z == 0xFF800000u) + (uint32_t)(q.w == 0xFF800000u);
+    }
+};
+
+// The part of a row the vector loop does not cover: the scalar head and tail of a row that is not
+// 16-byte aligned / not a whole number of vectors, and the penalised tokens from the history tables.
+template <int DT, class F>
+__device__ __forceinline__ void for_each_score_rest(const RowCtx &c, int head, int nvec, F &&fn) {
+    typedef Elem<DT> E;
+    const int V = c.V;
+    const int tail0 = head + nvec * E::PER_VEC;
+    for (int q = threadIdx.x; q < head + (V - tail0); q += NT) {
+        const int i = q < head ? q : tail0 + (q - head);
+        if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
+        fn(i, __fmul_rn(E::load(elem_ptr<DT>(c, i), 0), c.invT));
+    }
+    if (c.has_hist) {
+        for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
+            const int i = hist_id_of_rank(c, r);
+            const float x = E::load(elem_ptr<DT>(c, i), 0);
+            float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
+            av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(c.counts[r])));
+            av = __fsub_rn(av, c.p);
+            fn(i, __fmul_rn(av, c.invT));
+        }
+    }
+}
+
 // Calls fn(i, z_i) exactly once for every element of the row (each thread a share; any order).
 // Unpenalised elements come from 16-byte vector loads over the aligned middle of the row, two
 // loads in flight per thread, plus a scalar head and tail; penalised tokens (whose raw value is not
@@ -360,22 +503,50 @@ __device__ __forceinline__ void for_each_score(const RowCtx &c, F &&fn) {
                 if (!((m >> e) & 1u)) fn(i0 + e, __fmul_rn(E::get(q, e), c.invT));
         }
     }
-    const int tail0 = head + nvec * E::PER_VEC;
-    for (int q = threadIdx.x; q < head + (V - tail0); q += NT) {
-        const int i = q < head ? q : tail0 + (q - head);
-        if (c.has_hist && ((c.bitmap[i >> 5] >> (i & 31)) & 1u)) continue;
-        fn(i, __fmul_rn(E::load(elem_ptr<DT>(c, i), 0), c.invT));
-    }
-    if (c.has_hist) {
-        for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
-            const int i = hist_id_of_rank(c, r);
-            const float x = E::load(elem_ptr<DT>(c, i), 0);
-            float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
-            av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(c.counts[r])));
-            av = __fsub_rn(av, c.p);
-            fn(i, __fmul_rn(av, c.invT));
+    for_each_score_rest<DT>(c, head, nvec, fn);
+}
+
+// Pass 0 of the general path: the largest score key of the row and how many scores are finite.
+// Vectors without penalised tokens go through the packed maximum of the candidate path (the map
+// from raw value to score is increasing) with four loads in flight; the others element by element.
+template <int DT>
+__device__ __forceinline__ void pass0_max_count(const RowCtx &c, uint32_t &kbest, uint32_t &nfin) {
+    typedef Elem<DT> E;
+    typedef VecTest<DT> T;
+    const int V = c.V;
+    const uintptr_t addr = (uintptr_t)c.row;
+    int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
+    if (head > V) head = V;
+    const int nvec = (V - head) / E::PER_VEC;
+    const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
+    auto one = [&](int, float z) {
+        const uint32_t k = key_of(z);
+        kbest = k > kbest ? k : kbest;
+        nfin += (k >= KEY_MIN_FINITE && k < KEY_POS_INF);
+    };
+    for (int v0 = threadIdx.x; v0 < nvec; v0 += 4 * NT) {
+        uint4 q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) q[u] = (v0 + u * NT < nvec) ? __ldg(vec_ptr<DT>(c, vp, v0 + u * NT)) : T::fill();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = v0 + u * NT;
+            if (v >= nvec) break;
+            const int i0 = head + v * E::PER_VEC;
+            uint32_t m = 0;
+            if (c.has_hist) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31) & ((1u << E::PER_VEC) - 1u);
+            if (m == 0) {
+                const uint32_t k = T::vmax_key(q[u], c.invT);
+                kbest = k > kbest ? k : kbest;
+                nfin += (uint32_t)E::PER_VEC - T::count_neginf(q[u]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < E::PER_VEC; ++e)
+                    if (!((m >> e) & 1u)) one(i0 + e, __fmul_rn(E::get(q[u], e), c.invT));
+            }
         }
     }
+    for_each_score_rest<DT>(c, head, nvec, one);
 }
 
 // ------------------------------------------------------------------ history -> bitmap + counts
@@ -500,7 +671,6 @@ __device__ __forceinline__ void hist_clear(const HistBins &h) {
 }
 
 constexpr int GL_CAP = 2048;
-constexpr int SEL_ACC = NT;             // one accumulator per thread
 constexpr float BIN_SCALE = 32.0f;      // bins per unit of z
 
 struct RowParams {
@@ -596,40 +766,59 @@ __device__ int gather_if(BlockScratch &s, const HistBins &h, const RowCtx &c, F 
     return (int)s.list_cnt;
 }
 
-// On-chip: in h.list[0..n) (distinct composites within [lo, hi]) find the composite at which the
-// running total, taken from the largest composite down, first reaches `target` -- counting
-// elements (by_mass = false) or their masses.  Range-adaptive bins, repeated until a bin is one value.
-__device__ u64 list_resolve(BlockScratch &s, const HistBins &h, int n, bool by_mass, u64 target, u64 lo, u64 hi, float zmax) {
-    for (int pass = 0; pass < 8; ++pass) {
-        const u64 width = hi - lo;
-        const int shift = width < (u64)SEL_ACC ? 0 : bitlen64(width) - 9;
-        h.acc[threadIdx.x] = 0;
-        if (threadIdx.x == 0) s.found_digit = 0xFFFFFFFFu;
-        __syncthreads();
-        for (int i = threadIdx.x; i < n; i += NT) {
-            const u64 C = h.list[i];
-            if (C >= lo && C <= hi) {
-                const u64 v = by_mass ? mass_gen(__fsub_rn(unkey((uint32_t)(C >> 32)), zmax)) : 1ull;
-                atomicAdd(&h.acc[(hi - C) >> shift], v);
-            }
-        }
-        __syncthreads();
-        const u64 mine = h.acc[threadIdx.x];
-        u64 tot;
-        const u64 before = block_exscan_u64(s, mine, tot);
-        if (before < target && target <= before + mine) { s.found_digit = threadIdx.x; s.found_above = before; }
-        __syncthreads();
-        if (s.found_digit == 0xFFFFFFFFu) return lo;          // target beyond the list: keep all of it
-        const u64 b = s.found_digit;
-        target -= s.found_above;
-        const u64 nhi = hi - (b << shift);
-        if (shift == 0) return nhi;
-        const u64 span = (1ull << shift) - 1ull;
-        lo = (nhi - lo > span) ? nhi - span : lo;
-        hi = nhi;
-        __syncthreads();
+// On-chip: in h.list[0..n) (distinct composites, n <= GL_CAP) find the composite at which the running
+// total, taken from the largest composite down over those within [lo, hi], first reaches `target` --
+// counting elements (by_mass = false) or their masses.  The list is sorted in place (a bitonic network
+// over the next power of two, every thread a few compare-exchanges per step) and the totals are a
+// prefix sum over the sorted order: the cost does not depend on how the composites are spread, and
+// equal keys, which quantised logits produce in their hundreds, cost nothing extra.
+// (out of line, and given plain pointers only, so that it neither shapes the register allocation of
+// its callers nor forces their structures into local memory)
+__device__ __noinline__ u64 list_resolve(BlockScratch *sp, u64 *list, int n, bool by_mass, u64 target, u64 lo, u64 hi, float zmax) {
+    BlockScratch &s = *sp;
+    struct { u64 *list; } h = {list};
+    int P = 2;
+    while (P < n) P <<= 1;
+    for (int i = threadIdx.x; i < P; i += NT) {
+        const u64 C = i < n ? h.list[i] : 0ull;
+        h.list[i] = (C >= lo && C <= hi) ? C : 0ull;            // 0 sorts last and counts for nothing
     }
-    return lo;
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < (P >> 1); t += NT) {
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1)), l = i | j;
+                const u64 a = h.list[i], b2 = h.list[l];
+                const bool desc = (i & k) == 0;                  // final order: descending
+                if (desc ? a < b2 : a > b2) { h.list[i] = b2; h.list[l] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    // each thread owns a run of consecutive sorted entries
+    const int per = (P + NT - 1) / NT;
+    const int q0 = threadIdx.x * per, q1 = min(P, q0 + per);
+    u64 local = 0;
+    for (int q = q0; q < q1; ++q) {
+        const u64 C = h.list[q];
+        if (C) local += by_mass ? mass_gen(__fsub_rn(unkey((uint32_t)(C >> 32)), zmax)) : 1ull;
+    }
+    u64 tot;
+    u64 run = block_exscan_u64(s, local, tot);
+    if (threadIdx.x == 0) { s.bcast[3] = lo; }                   // target beyond the list: keep all of it
+    __syncthreads();
+    if (run < target && target <= run + local) {
+        for (int q = q0; q < q1; ++q) {
+            const u64 C = h.list[q];
+            if (!C) break;
+            run += by_mass ? mass_gen(__fsub_rn(unkey((uint32_t)(C >> 32)), zmax)) : 1ull;
+            if (run >= target) { s.bcast[3] = C; break; }
+        }
+    }
+    __syncthreads();
+    const u64 res = s.bcast[3];
+    __syncthreads();
+    return res;
 }
 
 // Exact cut inside the row: the composite at which the running total (count or mass, from the top of
@@ -675,7 +864,7 @@ __device__ u64 resolve_cut(BlockScratch &s, const HistBins &h, const RowCtx &c, 
     }
     if (n > GL_CAP) return lo > floorC ? lo : floorC;        // not reachable: composites are distinct
     if (n < 1) return floorC;
-    return list_resolve(s, h, n, by_mass, rel, lo, hi, zmax);
+    return list_resolve(&s, h.list, n, by_mass, rel, lo, hi, zmax);
 }
 
 template <int DT>
@@ -684,11 +873,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const int V = c.V;
     // pass 0: the largest key and the number of finite scores
     uint32_t kbest = 0, nfin_local = 0;
-    for_each_score<DT>(c, [&](int, float z) {
-        const uint32_t k = key_of(z);
-        kbest = k > kbest ? k : kbest;
-        nfin_local += (k >= KEY_MIN_FINITE && k < KEY_POS_INF);
-    });
+    pass0_max_count<DT>(c, kbest, nfin_local);
     const uint32_t kmax = (uint32_t)block_max_u64(s, kbest);
     const u64 n_fin = block_sum_u64(s, nfin_local);
     const float zmax = unkey(kmax);
@@ -1043,113 +1228,6 @@ __device__ int cand_compact(BlockScratch &s, const CandSmem &cs, int n, uint32_t
     __syncthreads();
     return (int)s.cand_cnt;
 }
-
-// Vector pre-test per dtype, in the domain the test runs in.
-// 16-bit types: raw logits; the threshold is the smallest raw value whose score has key >= tau
-// (packed twice).  x -> fl32(x * invT) is increasing, strictly so on distinct 16-bit values unless
-// the product leaves the fp32 range, so a compare of raw values is a superset of the key test.
-// fp32: scores; the threshold is unkey(tau).
-struct Bf16Packed {
-    typedef __nv_bfloat162 H2;
-    static constexpr uint32_t LO = 0x0080u, HI = 0xFF7Fu, NEG_INF = 0xFF80u;    // order codes of the finite range; -inf pattern
-    static __device__ __forceinline__ float widen(uint32_t bits) { return __uint_as_float(bits << 16); }
-    static __device__ __forceinline__ uint32_t truncate(float x) { return __float_as_uint(x) >> 16; }
-};
-struct F16Packed {
-    typedef __half2 H2;
-    static constexpr uint32_t LO = 0x0400u, HI = 0xFBFFu, NEG_INF = 0xFC00u;
-    static __device__ __forceinline__ float widen(uint32_t bits) { return __half2float(__ushort_as_half((unsigned short)bits)); }
-    static __device__ __forceinline__ uint32_t truncate(float x) { return __half_as_ushort(__float2half_rz(x)); }
-};
-template <int DT> struct VecTest;
-template <class P> struct VecTest16 {
-    typedef typename P::H2 H2;
-    static __device__ uint32_t raw_threshold(uint32_t tau_key, float invT) {
-        // order code of a 16-bit pattern (the analogue of the score key) and back
-        auto bits_of = [](uint32_t kk) { return (kk & 0x8000u) ? (kk & 0x7FFFu) : (~kk & 0xFFFFu); };
-        auto passes = [&](uint32_t kk) {
-            float x = P::widen(bits_of(kk));
-            return key_of(__fmul_rn(x, invT)) >= tau_key;
-        };
-        constexpr uint32_t LO = P::LO, HI = P::HI;             // the finite codes
-        // a guess from an approximate quotient, truncated to 16 bits: the answer is the guess or a
-        // neighbour, so the four codes around it are tried at once instead of one after another
-        const float xg = __fdividef(unkey(tau_key), invT);
-        const uint32_t b16 = P::truncate(xg) & 0xFFFFu;
-        uint32_t k16 = (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
-        k16 = k16 < LO + 2u ? LO + 2u : (k16 > HI - 1u ? HI - 1u : k16);
-        const bool p0 = passes(k16 - 2u), p1 = passes(k16 - 1u), p2 = passes(k16), p3 = passes(k16 + 1u);
-        uint32_t ans = 0;
-        if (p1 && !p0) ans = k16 - 1u;
-        else if (p2 && !p1) ans = k16;
-        else if (p3 && !p2) ans = k16 + 1u;
-        if (ans == 0) {
-            // not bracketed (an extreme temperature, or the ends of the range): a short walk
-            int it = 0;
-            while (it < 16 && k16 > LO && passes(k16)) { --k16; ++it; }
-            while (it < 32 && k16 < HI && !passes(k16)) { ++k16; ++it; }
-            const bool ok = passes(k16) && (k16 == LO || !passes(k16 - 1u));
-            ans = ok ? k16 : 0u;
-        }
-        const uint32_t b = ans ? bits_of(ans) : P::NEG_INF;    // not settled: let everything through
-        return b | (b << 16);
-    }
-    static __device__ __forceinline__ H2 vmax(const uint4 &q) {
-        H2 a = __hmax2(*reinterpret_cast<const H2 *>(&q.x), *reinterpret_cast<const H2 *>(&q.y));
-        H2 b2 = __hmax2(*reinterpret_cast<const H2 *>(&q.z), *reinterpret_cast<const H2 *>(&q.w));
-        return __hmax2(a, b2);
-    }
-    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float) {
-        return __hge2_mask(vmax(q), *reinterpret_cast<const H2 *>(&thr)) != 0u;
-    }
-    static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float) {
-        H2 m = vmax(q[0]);
-#pragma unroll
-        for (int u = 1; u < TILE_VECS; ++u) m = __hmax2(m, vmax(q[u]));
-        return __hge2_mask(m, *reinterpret_cast<const H2 *>(&thr)) != 0u;
-    }
-    // bit e set: raw element e >= the raw threshold (a superset of "score key >= tau")
-    static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float) {
-        const H2 t2 = *reinterpret_cast<const H2 *>(&thr);
-        const uint32_t r0 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.x), t2);
-        const uint32_t r1 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.y), t2);
-        const uint32_t r2 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.z), t2);
-        const uint32_t r3 = __hge2_mask(*reinterpret_cast<const H2 *>(&q.w), t2);
-        return ((r0 & 1u) | ((r0 >> 15) & 2u)) | (((r1 & 1u) | ((r1 >> 15) & 2u)) << 2) |
-               (((r2 & 1u) | ((r2 >> 15) & 2u)) << 4) | (((r3 & 1u) | ((r3 >> 15) & 2u)) << 6);
-    }
-    // key of the score of the vector's largest element (an element of the row)
-    static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) {
-        H2 m = vmax(q);
-        return key_of(__fmul_rn(fmaxf(__low2float(m), __high2float(m)), invT));
-    }
-    static __device__ __forceinline__ uint4 fill() { const uint32_t f = P::NEG_INF | (P::NEG_INF << 16); return make_uint4(f, f, f, f); }
-};
-template <> struct VecTest<ALBIREO_BF16> : VecTest16<Bf16Packed> {};
-template <> struct VecTest<ALBIREO_F16> : VecTest16<F16Packed> {};
-template <> struct VecTest<ALBIREO_F32> {
-    static __device__ uint32_t raw_threshold(uint32_t tau_key, float) { return __float_as_uint(unkey(tau_key)); }
-    static __device__ __forceinline__ float vmaxz(const uint4 &q, float invT) {
-        return fmaxf(fmaxf(__fmul_rn(__uint_as_float(q.x), invT), __fmul_rn(__uint_as_float(q.y), invT)),
-                     fmaxf(__fmul_rn(__uint_as_float(q.z), invT), __fmul_rn(__uint_as_float(q.w), invT)));
-    }
-    static __device__ __forceinline__ bool may_pass(const uint4 &q, uint32_t thr, float invT) {
-        return vmaxz(q, invT) >= __uint_as_float(thr);
-    }
-    static __device__ __forceinline__ bool any_may_pass(const uint4 (&q)[TILE_VECS], uint32_t thr, float invT) {
-        float m = vmaxz(q[0], invT);
-#pragma unroll
-        for (int u = 1; u < TILE_VECS; ++u) m = fmaxf(m, vmaxz(q[u], invT));
-        return m >= __uint_as_float(thr);
-    }
-    static __device__ __forceinline__ uint32_t elem_bits(const uint4 &q, uint32_t thr, float invT) {
-        const float t = __uint_as_float(thr);
-        return (uint32_t)(__fmul_rn(__uint_as_float(q.x), invT) >= t) | ((uint32_t)(__fmul_rn(__uint_as_float(q.y), invT) >= t) << 1) |
-               ((uint32_t)(__fmul_rn(__uint_as_float(q.z), invT) >= t) << 2) | ((uint32_t)(__fmul_rn(__uint_as_float(q.w), invT) >= t) << 3);
-    }
-    static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) { return key_of(vmaxz(q, invT)); }
-    static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
-};
 
 // bit e set: element e of the vector is unpenalised and its score has key >= tau
 template <int DT>
