@@ -1371,9 +1371,6 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
     }
 }
 
-// Starts the stream of a row that the candidate path will take: resets the per-row state, arms the
-// mbarriers and issues the first copies.  Called by the kernel before the history tables are
-// built, so that the first tiles arrive meanwhile; a block barrier must follow before any wait.
 // Threshold of the warm-up: a lower bound of the k-th largest of the block's per-thread maxima `mk`
 // (0: the thread has none), all of which lie in [kmin, kmax].  One pass: the maxima fall into
 // SEL_BINS value-linear bins (a monotone map of the key), each bin also keeps its smallest key; one
@@ -1417,6 +1414,9 @@ __device__ uint32_t warm_select(BlockScratch &s, const CandSmem &cs, uint32_t mk
     return s.found_digit;
 }
 
+// Starts the stream of a row: resets the per-row state, arms the mbarriers and issues the first
+// copies.  Called first thing in the kernel, before the row's parameters are loaded and the history
+// tables built, so that the first tiles arrive meanwhile; a block barrier must follow before any wait.
 template <int DT>
 __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c) {
     typedef Elem<DT> E;
