@@ -243,3 +243,22 @@ def test_argument_errors_launch_nothing(binding, sampler):
     sampler.albireo_sample(x)
     torch.cuda.synchronize()
     assert sampler.launch_count() == n0 + 1
+
+
+# ------------------------------------------------------------------ the largest supported vocabulary
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_maximum_vocabulary(binding, dtype, flags):
+    """V = ALBIREO_MAX_VOCAB with histories: the on-chip tables are at their largest (one CTA per SM)."""
+    V = binding.MAX_VOCAB
+    w = W.random_small(909, B=5, V=V, dtype=dtype)
+    w.num_top = 4
+    s = binding.Sampler(max_rows=8, max_vocab=V, max_history_total=int(w.history_ids.size))
+    try:
+        check(binding, s, w, flags=flags, allow_excused=1)
+        with pytest.raises(binding.AlbireoError):
+            big = torch.zeros((1, V + 8), dtype=torch.float32, device=s.device)
+            s.albireo_sample(big)
+    finally:
+        s.close()
