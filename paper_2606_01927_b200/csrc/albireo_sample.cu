@@ -117,21 +117,6 @@ __device__ __forceinline__ uint32_t race_word(uint64_t seed, uint32_t R, uint64_
     return wsel == 0 ? c0 : wsel == 1 ? c1 : wsel == 2 ? c2 : c3;
 }
 
-// all four words of the Philox block that serves tokens 4 blk .. 4 blk + 3
-__device__ __forceinline__ uint4 race_block(uint64_t seed, uint32_t R, uint64_t step, uint32_t blk) {
-    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
-    uint32_t c0 = blk, c1 = R, c2 = (uint32_t)step, c3 = (uint32_t)(step >> 32);
-    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
-#pragma unroll
-    for (int i = 0; i < 10; ++i) {
-        uint32_t h0 = __umulhi(M0, c0), l0 = M0 * c0;
-        uint32_t h1 = __umulhi(M1, c2), l1 = M1 * c2;
-        c0 = h1 ^ c1 ^ k0; c1 = l1; c2 = h0 ^ c3 ^ k1; c3 = l0;
-        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
-    }
-    return make_uint4(c0, c1, c2, c3);
-}
-
 // -ln(E) for E = -log1p(-v), v = (w + 1/2) 2^-32, in fp32.  The half of the range near
 // v = 1 is evaluated from 1 - v = (~w + 1/2) 2^-32 so both ends keep full relative accuracy.
 __device__ __forceinline__ float neg_log_exp1_f32(uint32_t w) {
@@ -636,6 +621,13 @@ __device__ int hist_id_of_rank(const RowCtx &c, uint32_t r) {
     return (w << 5) + (int)__fns(c.bitmap[w], 0, (int)rem + 1);
 }
 
+// -ln E of token i for the general path's race, out of line with plain arguments only: the long
+// Philox chain gets registers of its own and no structure of the caller is touched.
+__device__ __noinline__ float race_nle(uint64_t seed, uint32_t R, uint64_t step, const float *exp1_row, int i) {
+    if (exp1_row) return -logf(__ldg(exp1_row + i));
+    return neg_log_exp1_fast(race_word(seed, R, step, i));
+}
+
 // ------------------------------------------------------------------ general path: histogram selection
 //
 // For rows the candidate path does not take (top-p without top-k, no cuts at all, a top-k above
@@ -974,36 +966,77 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
 
     // final pass: mass of the kept set, its size, and the race.  An element whose score cannot
     // beat the thread's best even with the luckiest draw (-ln E <= 23 for the generator's words) is skipped.
+    // The race term is a long computation that only kept elements need, and in a wide kept set they
+    // are scattered over the lanes of a warp: running it in place would execute it for almost every
+    // element position with few lanes active.  So each thread queues its contenders in shared memory
+    // (a private queue, over the histograms, which are done with) and the warp works the queues off
+    // together whenever one of them runs full: then most lanes have an entry to work on.
     u64 S_local = 0, g_best = 0;
     uint32_t n_local = 0;
     float best_g = -3.0e38f;
     const uint32_t k2 = (uint32_t)(C2 >> 32);
     const int id2 = comp_idx(C2);
-    uint32_t blk_id = 0xFFFFFFFFu;                       // neighbouring tokens share a Philox block: keep the last one
-    uint4 blk = make_uint4(0, 0, 0, 0);
     const float *exp1_row = a.exp1 ? a.exp1 + (int64_t)b * a.exp1_stride : nullptr;
     const float luck = exp1_row ? 104.0f : 23.0f;        // largest -ln E: a table may hold any positive fp32
-    for_each_score<DT>(c, [&](int i, float z) {
+    have_hist = have_mass = false;
+    __syncthreads();
+    constexpr int RQ_DEPTH = 12;                         // 8 elements of a vector on top of at most 4 left over
+    u64 *rq = (u64 *)h.cnt + threadIdx.x;                // entry j of this thread at rq[j * NT]: 48 KiB in all
+    int qn = 0;
+    auto race_one = [&](int i, float d) {
+        if (d + luck >= best_g) {
+            const float g = d + race_nle(rp.seed, rp.R, a.step, exp1_row, i);
+            const u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
+            if (G > g_best) { g_best = G; best_g = g; }
+        }
+    };
+    auto see = [&](int i, float z, bool may_queue) {
         const uint32_t k = key_of(z);
         if (k > k2 || (k == k2 && i <= id2)) {
             const float d = __fsub_rn(z, zmax);
             S_local += mass_gen(d);
             n_local += 1;
             if (d + luck >= best_g) {
-                float nle;
-                if (exp1_row) nle = -logf(__ldg(exp1_row + i));
-                else {
-                    if (((uint32_t)i >> 2) != blk_id) { blk_id = (uint32_t)i >> 2; blk = race_block(rp.seed, rp.R, a.step, blk_id); }
-                    const int wsel = i & 3;
-                    const uint32_t w = wsel == 0 ? blk.x : wsel == 1 ? blk.y : wsel == 2 ? blk.z : blk.w;
-                    nle = neg_log_exp1_fast(w);
-                }
-                const float g = d + nle;
-                const u64 G = ((u64)orderable_f32(g) << 32) | (uint32_t)(~(uint32_t)i);
-                if (G > g_best) { g_best = G; best_g = g; }
+                if (may_queue && qn < RQ_DEPTH) { rq[qn * NT] = ((u64)__float_as_uint(d) << 32) | (uint32_t)i; ++qn; }
+                else race_one(i, d);
             }
         }
-    });
+    };
+    // called by whole warps: works the queues down until none holds more than `leave`
+    auto drain = [&](int leave) {
+        while (__any_sync(0xFFFFFFFFu, qn > leave)) {
+            if (qn > 0) { --qn; const u64 e = rq[qn * NT]; race_one((int)(uint32_t)e, __uint_as_float((uint32_t)(e >> 32))); }
+        }
+    };
+    {
+        typedef Elem<DT> E;
+        const uintptr_t addr = (uintptr_t)c.row;
+        int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
+        if (head > V) head = V;
+        const int nvec = (V - head) / E::PER_VEC;
+        const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
+        for (int base = 0; base < nvec; base += 2 * NT) {            // the same trip count in every thread
+            const int v0 = base + (int)threadIdx.x, v1 = v0 + NT;
+            const uint4 q0 = v0 < nvec ? __ldg(vec_ptr<DT>(c, vp, v0)) : make_uint4(0, 0, 0, 0);
+            const uint4 q1 = v1 < nvec ? __ldg(vec_ptr<DT>(c, vp, v1)) : q0;
+#pragma unroll 1
+            for (int u = 0; u < 2; ++u) {
+                const int v = u ? v1 : v0;
+                if (v < nvec) {
+                    const uint4 &q = u ? q1 : q0;
+                    const int i0 = head + v * E::PER_VEC;
+                    uint32_t m = 0;
+                    if (c.has_hist) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+#pragma unroll
+                    for (int e = 0; e < E::PER_VEC; ++e)
+                        if (!((m >> e) & 1u)) see(i0 + e, __fmul_rn(E::get(q, e), c.invT), true);
+                }
+                drain(RQ_DEPTH - E::PER_VEC);
+            }
+        }
+        for_each_score_rest<DT>(c, head, nvec, [&](int i, float z) { see(i, z, true); });
+        drain(0);
+    }
     const u64 S_fx = block_sum_u64(s, S_local);
     const u64 n_keep = block_sum_u64(s, n_local);
     const u64 G = block_max_u64(s, g_best);
