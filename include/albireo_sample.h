@@ -15,7 +15,8 @@
  *   x      = logits widened to fp32
  *   c_t    = occurrences of token t in the row's history (ids outside [0,V) ignored)
  *   a_t    = x_t                              if c_t == 0
- *          = ((x_t > 0 ? x_t / r : x_t * r) - f * c_t) - p   otherwise (fp32, one rounding per op)
+ *          = ((x_t > 0 ? x_t / r : x_t * r) - f * c_t) - p   otherwise (fp32, one rounding per op;
+ *            with ext->history_output_start see there)
  *   z_t    = a_t * (1 / T)   (fp32; T <= 0 means greedy: top_k = 1 on a_t, other cuts ignored)
  *   order  = ids sorted by (z descending, id ascending); -0.0 sorts below +0.0
  *   top-k  : keep the first min(k, #finite z)          (k <= 0 or k >= V: off)
@@ -124,6 +125,15 @@ typedef struct albireo_sample_ext {
        of 16 (ALBIREO_EUNSUPPORTED otherwise).  0 or 1: rows are contiguous.                */
     int32_t num_segments;
     int64_t segment_stride_elems;
+
+    /* Prompt / output split of the histories (the per-sequence sampling metadata of section 3.1
+       keeps prompt and generated tokens apart).  history_output_start[b] = number of leading ids
+       of row b's history that are the prompt; the rest is generated output.  The repetition
+       penalty then applies to a token seen in either part, the frequency penalty uses the
+       occurrences in the output alone and the presence penalty applies only if there is one:
+       a = rep(x); a -= f * c_out; if (c_out > 0) a -= p.  Values are clamped to [0, length].
+       NULL: every id counts as output (the three penalties share one history).             */
+    const int32_t *history_output_start; /* [B] device, or NULL                              */
 } albireo_sample_ext_t;
 
 /*

@@ -17,6 +17,10 @@
  *   2. count history occurrences per token id (ids outside [0,V) ignored);
  *   3. for tokens with count > 0: a = x>0 ? x/r : x*r ; a -= f*count ; a -= p
  *      (each step one rounded fp32 operation);
+ *      with the history split into prompt and generated output (`out_start`: where the output begins
+ *      in the row's history) the repetition penalty looks at both parts, the frequency and presence
+ *      penalties at the output alone: a = rep(x) for a token seen anywhere; a -= f*c_out; and
+ *      a -= p only if c_out > 0 (c_out: occurrences in the output);
  *   4. T == 0 (or < 0): greedy == top_k 1 with no scaling; else z = a * (1/T) in fp32;
  *   5. sort all ids by (order-preserving key of z descending, id ascending);
  *   6. top-k: keep the first min(k, #finite);  7. min-p: keep z - zmax >= ln(min_p);
@@ -154,24 +158,33 @@ typedef struct {
  * Returns 1 if the row is greedy.
  */
 static int row_scores_and_order(const void *logits, int32_t dtype, int64_t row_pos, int32_t V,
-                                const int32_t *hist, int32_t hist_len, const row_params_t *rp,
+                                const int32_t *hist, int32_t hist_len, int32_t out_start,
+                                const row_params_t *rp,
                                 int32_t *counts, float *z, sort_item_t *order)
 {
+    if (out_start < 0) out_start = 0;
+    if (out_start > hist_len) out_start = hist_len;
     /* 1. widen */
     for (int32_t i = 0; i < V; ++i) z[i] = load_logit(logits, dtype, row_pos + i);
-    /* 2. counts */
-    for (int32_t j = 0; j < hist_len; ++j) {
+    /* 2. counts: counts[t] = occurrences in the output part; a token seen only in the prompt is
+       marked with -1 (seen, zero output occurrences) */
+    for (int32_t j = out_start; j < hist_len; ++j) {
         int32_t t = hist[j];
         if (t >= 0 && t < V) counts[t] += 1;
     }
+    for (int32_t j = 0; j < out_start; ++j) {
+        int32_t t = hist[j];
+        if (t >= 0 && t < V && counts[t] == 0) counts[t] = -1;
+    }
     /* 3. penalties, one rounded fp32 operation per line */
     for (int32_t i = 0; i < V; ++i) {
-        if (counts[i] > 0) {
+        if (counts[i] != 0) {
+            int32_t c_out = counts[i] > 0 ? counts[i] : 0;
             float a = z[i];
             if (a > 0.0f) a = a / rp->r; else a = a * rp->r;
-            float t = rp->f * (float)counts[i];
+            float t = rp->f * (float)c_out;
             a = a - t;
-            a = a - rp->p;
+            if (c_out > 0) a = a - rp->p;
             z[i] = a;
         }
     }
@@ -308,6 +321,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                           const int32_t *hist_ids, const int32_t *hist_off,
                           const uint64_t *seeds, uint64_t step, uint32_t row_base,
                           const float *exp1 /* [B, V] Exp(1) variates, or NULL */,
+                          const int32_t *out_start /* [B] where the output begins in each history, or NULL: 0 */,
                           int32_t row_begin, int32_t row_end,
                           albireo_oracle_row_t *rows_out,
                           int32_t topk_cap, int32_t *topk_ids,
@@ -327,7 +341,8 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
         load_params(b, temperature, top_k, top_p, min_p, rep, pres, freq, seeds, &rp);
         const int32_t *h = NULL; int32_t hl = 0;
         if (hist_ids && hist_off) { h = hist_ids + hist_off[b]; hl = hist_off[b + 1] - hist_off[b]; }
-        int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl, &rp, counts, z, order);
+        int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl,
+                                          out_start ? out_start[b] : 0, &rp, counts, z, order);
         albireo_oracle_row_t *o = &rows_out[b];
         row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step,
                          exp1 ? exp1 + (int64_t)b * V : NULL, 0.0, 0.0, o, e);
@@ -365,7 +380,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
                                const float *min_p, const float *rep, const float *pres, const float *freq,
                                const int32_t *hist_ids, const int32_t *hist_off,
                                const uint64_t *seeds, uint64_t step, uint32_t row_base,
-                               const float *exp1,
+                               const float *exp1, const int32_t *out_start,
                                int32_t b, double ln_min_p_shift, double top_p_shift,
                                albireo_oracle_row_t *row_out, int32_t *sorted_ids, float *sorted_z,
                                double *sorted_g)
@@ -380,7 +395,8 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
     load_params(b, temperature, top_k, top_p, min_p, rep, pres, freq, seeds, &rp);
     const int32_t *h = NULL; int32_t hl = 0;
     if (hist_ids && hist_off) { h = hist_ids + hist_off[b]; hl = hist_off[b + 1] - hist_off[b]; }
-    int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl, &rp, counts, z, order);
+    int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl,
+                                      out_start ? out_start[b] : 0, &rp, counts, z, order);
     const float *exp1_row = exp1 ? exp1 + (int64_t)b * V : NULL;
     row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, exp1_row,
                      ln_min_p_shift, top_p_shift, row_out, e);
@@ -401,7 +417,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
 /* the penalised, temperature-scaled scores z of one row (steps 1-4), for pins */
 int albireo_oracle_row_scores(const void *logits, int32_t V, int32_t dtype,
                               float T, float r, float p, float f,
-                              const int32_t *hist, int32_t hist_len, float *z_out)
+                              const int32_t *hist, int32_t hist_len, int32_t out_start, float *z_out)
 {
     if (!logits || !z_out || V < 1) return -1;
     sort_item_t *order = (sort_item_t *)malloc(sizeof(sort_item_t) * (size_t)V);
@@ -409,7 +425,7 @@ int albireo_oracle_row_scores(const void *logits, int32_t V, int32_t dtype,
     if (!order || !counts) { free(order); free(counts); return -1; }
     row_params_t rp; memset(&rp, 0, sizeof rp);
     rp.T = T; rp.r = r; rp.p = p; rp.f = f; rp.top_p = 1.0f;
-    row_scores_and_order(logits, dtype, 0, V, hist, hist_len, &rp, counts, z_out, order);
+    row_scores_and_order(logits, dtype, 0, V, hist, hist_len, out_start, &rp, counts, z_out, order);
     free(order); free(counts);
     return 0;
 }

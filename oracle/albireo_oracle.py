@@ -94,6 +94,7 @@ def _common_args(w):
         _ptr(w.history_ids, np.int32), _ptr(w.history_offsets, np.int32),
         _ptr(w.seeds, np.uint64), C.c_uint64(w.step), C.c_uint32(w.row_base),
         _ptr(getattr(w, "exp1", None), np.float32),
+        _ptr(getattr(w, "output_start", None), np.int32),
     ]
 
 
@@ -169,7 +170,7 @@ def row_shifted(w, b: int, ln_min_p_shift: float = 0.0, top_p_shift: float = 0.0
     return res[0], ids, zs, gs
 
 
-def row_scores(logits_row: np.ndarray, dtype: int, T=1.0, r=1.0, p=0.0, f=0.0, history=None) -> np.ndarray:
+def row_scores(logits_row: np.ndarray, dtype: int, T=1.0, r=1.0, p=0.0, f=0.0, history=None, output_start: int = 0) -> np.ndarray:
     """Steps 1-4 (widen, penalties, temperature) of one row; returns z as float32[V]."""
     L = lib()
     V = logits_row.shape[0]
@@ -178,7 +179,7 @@ def row_scores(logits_row: np.ndarray, dtype: int, T=1.0, r=1.0, p=0.0, f=0.0, h
     rc = L.albireo_oracle_row_scores(
         _ptr(np.ascontiguousarray(logits_row), np.float32 if dtype == 0 else np.uint16),
         C.c_int32(V), C.c_int32(dtype), C.c_float(T), C.c_float(r), C.c_float(p), C.c_float(f),
-        _ptr(h, np.int32), C.c_int32(0 if h is None else h.size), z.ctypes.data_as(C.c_void_p))
+        _ptr(h, np.int32), C.c_int32(0 if h is None else h.size), C.c_int32(output_start), z.ctypes.data_as(C.c_void_p))
     if rc != 0:
         raise RuntimeError("albireo_oracle_row_scores failed")
     return z

@@ -51,6 +51,7 @@ class SampleExt(C.Structure):
         ("backfill_ids", C.c_void_p), ("backfill_index", C.c_void_p), ("backfill_len", C.c_int64),
         ("feedback_ring", C.c_void_p), ("feedback_cap", C.c_int64), ("feedback_head", C.c_int64),
         ("num_segments", C.c_int32), ("segment_stride_elems", C.c_int64),
+        ("history_output_start", C.c_void_p),
     ]
 
 
@@ -203,7 +204,7 @@ class Sampler:
                        want_status=False, flags: int = 0, B: Optional[int] = None, V: Optional[int] = None,
                        exp1: Optional[torch.Tensor] = None, backfill_ids: Optional[torch.Tensor] = None,
                        backfill_index: Optional[torch.Tensor] = None, feedback_ring: Optional[torch.Tensor] = None,
-                       feedback_head: int = 0) -> SampleOutputs:
+                       feedback_head: int = 0, output_start: Optional[torch.Tensor] = None) -> SampleOutputs:
         """Device-resident call: all tensors on ``self.device``; asynchronous on ``stream``.
 
         ``exp1`` (float32 ``[B, V]``) replaces the counter-based draw by pre-generated Exp(1)
@@ -238,6 +239,8 @@ class Sampler:
             ext.num_segments = nseg
             ext.segment_stride_elems = logits.stride(0)
             ext.row_stride_elems = row_stride
+        if output_start is not None:
+            ext.history_output_start = _dp(output_start, torch.int32, "cuda")
         if exp1 is not None:
             if exp1.dtype != torch.float32 or exp1.dim() != 2 or exp1.stride(1) != 1 or exp1.device != dev:
                 raise ValueError("exp1 must be a float32 [B, V] tensor on the logits' device")
@@ -368,6 +371,8 @@ def workload_tensors(w, device, pinned: bool = False) -> dict:
         extra["exp1"] = conv(w.exp1)
     if getattr(w, "backfill_index", None) is not None:
         extra["backfill_index"] = conv(w.backfill_index)
+    if getattr(w, "output_start", None) is not None:
+        extra["output_start"] = conv(w.output_start)
     return dict(
         **extra,
         logits=logits, temperature=conv(w.temperature), top_k=conv(w.top_k), top_p=conv(w.top_p),

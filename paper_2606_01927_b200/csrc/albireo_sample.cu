@@ -76,6 +76,7 @@ struct SampleArgs {
     uint32_t *out_row_status;
     int32_t elem_size;          // host side only: bytes per logit
     int32_t nstages;            // ring depth chosen by the host for this launch
+    const int32_t *out_start;   // per row: where the generated output begins in the history, or null: at 0
     const float *exp1;          // pre-generated Exp(1) variates [B, exp1_stride], or null: counter-based draw
     int64_t exp1_stride;
     int32_t *backfill_ids;      // early feedback: next iteration's input ids, or null
@@ -244,13 +245,16 @@ __device__ __forceinline__ uint32_t hist_rank(const RowCtx &c, int i) {
 }
 
 // penalties: each line is one rounded fp32 operation
-__device__ __forceinline__ float penalise(const RowCtx &c, int i, float x) {
-    uint32_t cnt = c.counts[hist_rank(c, i)];
+// the penalties of a token seen in the history, `cnt` of its occurrences in the generated output
+// (all of them when the history is not split; 0 for a token seen in the prompt only)
+__device__ __forceinline__ float penalise_counted(const RowCtx &c, float x, uint32_t cnt) {
     float a = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
-    float t = __fmul_rn(c.f, __uint2float_rn(cnt));
-    a = __fsub_rn(a, t);
-    a = __fsub_rn(a, c.p);
+    a = __fsub_rn(a, __fmul_rn(c.f, __uint2float_rn(cnt)));
+    if (cnt) a = __fsub_rn(a, c.p);
     return a;
+}
+__device__ __forceinline__ float penalise(const RowCtx &c, int i, float x) {
+    return penalise_counted(c, x, c.counts[hist_rank(c, i)]);
 }
 
 template <int DT> struct Elem;
@@ -451,9 +455,7 @@ __device__ __forceinline__ void for_each_score_rest(const RowCtx &c, int head, i
         for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
             const int i = hist_id_of_rank(c, r);
             const float x = E::load(elem_ptr<DT>(c, i), 0);
-            float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
-            av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(c.counts[r])));
-            av = __fsub_rn(av, c.p);
+            const float av = penalise_counted(c, x, c.counts[r]);
             fn(i, __fmul_rn(av, c.invT));
         }
     }
@@ -560,7 +562,8 @@ __device__ uint32_t block_exscan_u32(BlockScratch &s, uint32_t v, uint32_t &tota
 
 // Builds the per-row penalty tables.  Returns false (penalties skipped) if the distinct
 // ids fit neither on chip nor in the caller's workspace.
-__device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, const int32_t *ids, int len,
+// Ids before position out_start are the prompt: they set their bit (repetition penalty) but are not counted.
+__device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, const int32_t *ids, int len, int out_start,
                               uint32_t *ws, int64_t ws_cap, int64_t ws_off) {
     const int V = c.V;
     const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
@@ -602,10 +605,10 @@ __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, co
     for (uint32_t u = threadIdx.x; u < U; u += NT) cnt[u] = 0;
     __syncthreads();
 #pragma unroll
-    for (int q = 0; q < KEEP; ++q) { const int t = mine[q]; if (t >= 0 && t < V) atomicAdd(&cnt[hist_rank(c, t)], 1u); }
+    for (int q = 0; q < KEEP; ++q) { const int t = mine[q]; if (t >= 0 && t < V && (int)threadIdx.x + q * NT >= out_start) atomicAdd(&cnt[hist_rank(c, t)], 1u); }
     for (int j = threadIdx.x + KEEP * NT; j < len; j += NT) {
         int t = __ldg(ids + j);
-        if (t >= 0 && t < V) atomicAdd(&cnt[hist_rank(c, t)], 1u);
+        if (t >= 0 && t < V && j >= out_start) atomicAdd(&cnt[hist_rank(c, t)], 1u);
     }
     __syncthreads();
     return true;
@@ -1734,9 +1737,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             const int i = hist_id_of_rank(c, r);
             const float x = E::load(elem_ptr<DT>(c, i), 0);
             const uint32_t cntv = c.counts[r];
-            float av = (x > 0.0f) ? __fdiv_rn(x, c.r) : __fmul_rn(x, c.r);
-            av = __fsub_rn(av, __fmul_rn(c.f, __uint2float_rn(cntv)));
-            av = __fsub_rn(av, c.p);
+            const float av = penalise_counted(c, x, cntv);
             const uint32_t key = key_of(__fmul_rn(av, c.invT));
             if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
         }
@@ -1840,7 +1841,8 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     if (a.hist_ids && a.hist_off) {
         const int o0 = a.hist_off[b], o1 = a.hist_off[b + 1];
         if (o1 > o0) {
-            bool ok = build_history(s, hs, c, a.hist_ids + o0, o1 - o0, a.ws_counts, a.ws_counts_cap, (int64_t)o0);
+            const int ostart = a.out_start ? a.out_start[b] : 0;
+            bool ok = build_history(s, hs, c, a.hist_ids + o0, o1 - o0, ostart, a.ws_counts, a.ws_counts_cap, (int64_t)o0);
             c.has_hist = ok;
             if (!ok) out.status |= ALBIREO_ROW_HISTORY_OVERFLOW;
         }
@@ -1948,6 +1950,7 @@ int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, cons
         }
         a.nseg = (int32_t)t; a.seg_stride = ext->segment_stride_elems;
     } else if (ext->num_segments < 0) { *why = "num_segments is negative"; return ALBIREO_EINVAL; }
+    a.out_start = ext->history_output_start;
     if (ext->exp1) {
         if (ext->exp1_stride_elems != 0 && ext->exp1_stride_elems < V) { *why = "exp1 row stride smaller than V"; return ALBIREO_EINVAL; }
         if ((uintptr_t)ext->exp1 % 4) { *why = "exp1 not 4-byte aligned"; return ALBIREO_EINVAL; }
@@ -2127,7 +2130,7 @@ extern "C" int albireo_sample_host(albireo_sampler_t *h, const void *logits, int
     if (ext && ext->struct_size != sizeof(albireo_sample_ext_t)) { set_err(h, "ext->struct_size mismatch%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->row_stride_elems != 0 && ext->row_stride_elems != V) { set_err(h, "host entry needs dense rows%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->dbg_cap > 0) { set_err(h, "host entry has no debug output%s", ""); return ALBIREO_EINVAL; }
-    if (ext && (ext->exp1 || ext->backfill_ids || ext->feedback_ring || ext->num_segments > 1)) { set_err(h, "host entry takes no exp1 table, no early-feedback targets and no rows in pieces%s", ""); return ALBIREO_EINVAL; }
+    if (ext && (ext->exp1 || ext->backfill_ids || ext->feedback_ring || ext->num_segments > 1 || ext->history_output_start)) { set_err(h, "host entry takes no exp1 table, no early-feedback targets, no rows in pieces and no history split%s", ""); return ALBIREO_EINVAL; }
     const size_t base = albireo_sample_workspace_bytes(h->max_rows, h->max_vocab, h->max_history_total);
     if (h->workspace_bytes < base + albireo_sample_host_staging_bytes(h->max_rows, h->max_vocab, h->max_history_total)) {
         set_err(h, "workspace given to init has no staging space%s", ""); return ALBIREO_EINVAL;

@@ -51,7 +51,9 @@ class Workload:
     a float32 ``[B, V]`` table of Exp(1) variates read instead of the counter-based
     generator.  ``backfill_index`` (int32 ``[B]``, -1 = skip) says where in the next
     iteration's input-id tensor of ``backfill_len`` entries each row's token goes
-    (early feedback, §5.2).
+    (early feedback, §5.2).  ``output_start`` (int32 ``[B]``) splits each history into prompt
+    (the first ``output_start[b]`` ids) and generated output (the rest): the repetition penalty then
+    looks at both, the presence and frequency penalties at the output alone.
     """
 
     name: str
@@ -75,6 +77,7 @@ class Workload:
     exp1: Optional[np.ndarray] = None
     backfill_index: Optional[np.ndarray] = None
     backfill_len: int = 0
+    output_start: Optional[np.ndarray] = None
     notes: dict = field(default_factory=dict)
 
     @property
@@ -115,7 +118,8 @@ class Workload:
             presence_penalty=cut(self.presence_penalty), frequency_penalty=cut(self.frequency_penalty),
             history_ids=hid, history_offsets=hoff, seeds=cut(self.seeds), step=self.step,
             row_base=self.row_base + lo, num_top=self.num_top, exp1=cut(self.exp1),
-            backfill_index=cut(self.backfill_index), backfill_len=self.backfill_len, notes=dict(self.notes))
+            backfill_index=cut(self.backfill_index), backfill_len=self.backfill_len,
+            output_start=cut(self.output_start), notes=dict(self.notes))
 
 
 # --------------------------------------------------------------------------- helpers
@@ -345,5 +349,22 @@ def with_backfill(w: Workload, seed: int = 11, slack: int = 3) -> Workload:
     idx = rng.permutation(out.backfill_len)[: w.B].astype(np.int32)
     idx[rng.random(w.B) < 0.125] = -1
     out.backfill_index = idx
+    out.notes = dict(w.notes)
+    return out
+
+
+def with_split_history(w: Workload, seed: int = 13) -> Workload:
+    """The same workload with every history split at a random point into prompt and output
+    (a few rows all prompt, a few all output)."""
+    import copy
+    out = copy.copy(w)
+    out.name = w.name + "_split"
+    rng = np.random.Generator(np.random.PCG64(seed))
+    lens = np.diff(w.history_offsets.astype(np.int64))
+    start = np.floor(rng.random(w.B) * (lens + 1)).astype(np.int32)
+    pick = rng.random(w.B)
+    start[pick < 0.1] = 0
+    start[pick > 0.9] = lens[pick > 0.9].astype(np.int32)
+    out.output_start = start
     out.notes = dict(w.notes)
     return out

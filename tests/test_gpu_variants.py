@@ -274,3 +274,36 @@ def test_sequence_parallel_step_on_one_rank(binding, sampler):
         assert np.abs(lp.cpu().numpy()[tok.cpu().numpy() == ref.tokens] - ref.logprobs[tok.cpu().numpy() == ref.tokens]).max() < 1e-4
     finally:
         dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------ prompt / output split of the histories
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_split_history_small(binding, sampler, dtype, flags):
+    w = W.with_split_history(W.random_small(601, B=48, V=4099, dtype=dtype))
+    w.num_top = 4
+    check(binding, sampler, w, flags=flags)
+
+
+def test_split_history_full_vocabulary_and_limits(binding, sampler):
+    base = W.config3(B=24)
+    w = W.with_split_history(base)
+    g, ref = check(binding, sampler, w)
+    # all-output split == no split, bit for bit
+    w0 = W.config3(B=24)
+    w0.output_start = np.zeros(w0.B, dtype=np.int32)
+    a = run(binding, sampler, w0)
+    b = run(binding, sampler, W.config3(B=24))
+    assert (a["tokens"] == b["tokens"]).all() and (a["logprobs"] == b["logprobs"]).all()
+    # out-of-range values are clamped to [0, length]
+    w1 = W.config3(B=24)
+    w1.output_start = np.full(w1.B, -5, dtype=np.int32)
+    c = run(binding, sampler, w1)
+    assert (c["tokens"] == b["tokens"]).all()
+    w2 = W.config3(B=24)
+    w2.output_start = np.full(w2.B, 10**6, dtype=np.int32)
+    w3 = W.config3(B=24)
+    w3.output_start = np.diff(w3.history_offsets).astype(np.int32)
+    d, e = run(binding, sampler, w2), run(binding, sampler, w3)
+    assert (d["tokens"] == e["tokens"]).all() and (d["logprobs"] == e["logprobs"]).all()

@@ -534,3 +534,55 @@ def test_exp1_table_draw_frequencies():
     obs = np.bincount(tok, minlength=V)
     p = np.exp(x.astype(np.float64)); p /= p.sum()
     assert scipy.stats.chisquare(obs, p * N).pvalue > 1e-4
+
+
+# ------------------------------------------------------------------ prompt / output split of the history
+
+def test_split_history_elementwise_and_limits():
+    """Repetition looks at prompt and output, presence and frequency at the output alone; each step
+    one IEEE fp32 operation, recomputed here from the two parts' own tallies."""
+    rng = np.random.default_rng(51)
+    V = 400
+    x = (rng.standard_normal(V) * 3).astype(np.float32)
+    hist = rng.integers(-2, V + 2, size=600)
+    r, p, f, T = np.float32(1.25), np.float32(0.6), np.float32(0.2), np.float32(0.8)
+    inv_T = np.float32(1.0) / T
+    valid = lambda h: h[(h >= 0) & (h < V)]
+    for start in (0, 1, 250, 599, 600):
+        z = O.row_scores(x, W.F32, T=float(T), r=float(r), p=float(p), f=float(f), history=hist, output_start=start)
+        c_any = np.bincount(valid(hist), minlength=V)
+        c_out = np.bincount(valid(hist[start:]), minlength=V)
+        assert start != 250 or ((c_any > 0) & (c_out == 0)).sum() >= 5            # prompt-only tokens exist
+        for i in range(V):
+            a = x[i]
+            if c_any[i] > 0:
+                a = a / r if a > 0 else a * r
+                a = a - f * np.float32(c_out[i])
+                if c_out[i] > 0:
+                    a = a - p
+            assert np.float32(a * inv_T) == z[i], (start, i)
+    # limits: everything output == no split; everything prompt == repetition penalty alone
+    z_all_out = O.row_scores(x, W.F32, T=float(T), r=float(r), p=float(p), f=float(f), history=hist, output_start=0)
+    z_plain = O.row_scores(x, W.F32, T=float(T), r=float(r), p=float(p), f=float(f), history=hist)
+    assert (z_all_out.view(np.uint32) == z_plain.view(np.uint32)).all()
+    z_all_prompt = O.row_scores(x, W.F32, T=float(T), r=float(r), p=float(p), f=float(f), history=hist, output_start=600)
+    z_rep_only = O.row_scores(x, W.F32, T=float(T), r=float(r), p=0.0, f=0.0, history=hist)
+    assert (z_all_prompt.view(np.uint32) == z_rep_only.view(np.uint32)).all()
+
+
+def test_split_history_through_the_batch_entry():
+    w = W.with_split_history(W.random_small(53, B=12, V=300, dtype=W.F32))
+    assert w.output_start is not None and (w.output_start >= 0).all()
+    got = O.sample(w, kept_cap=8)
+    # the same rows one by one, each with its own split handed to the single-row score routine
+    for b in range(w.B):
+        o = w.history_offsets
+        z = O.row_scores(w.logits[b], W.F32, T=float(w.temperature[b]) if w.temperature[b] > 0 else 1.0,
+                         r=float(w.repetition_penalty[b]), p=float(w.presence_penalty[b]),
+                         f=float(w.frequency_penalty[b]), history=w.history_ids[o[b]:o[b + 1]],
+                         output_start=int(w.output_start[b]))
+        assert got.kept_ids[b][0] == int(np.lexsort((np.arange(w.V), -z.astype(np.float64)))[0])
+    # and the split matters: some row's token or logprob differs from the unsplit run
+    w0 = W.random_small(53, B=12, V=300, dtype=W.F32)
+    base = O.sample(w0)
+    assert (base.tokens != got.tokens).any() or (base.logprobs != got.logprobs).any()
