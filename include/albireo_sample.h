@@ -65,6 +65,10 @@ enum {
 
 /* flags of albireo_sample_ext_t.flags */
 #define ALBIREO_FLAG_FORCE_GENERAL 1u /* testing: send every row down the general path     */
+#define ALBIREO_FLAG_TOPK_KEEP_TIES 2u /* top-k keeps every score not below the k-th largest
+                                         (what masking "logits < k-th value" gives) instead of
+                                         exactly k ids; equal means equal in the order, so -0.0
+                                         stays below +0.0; greedy rows are not affected          */
 
 /*
  * Optional arguments of albireo_sample (pass NULL for all defaults).  Zero-initialise,

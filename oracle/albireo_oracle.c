@@ -23,7 +23,9 @@
  *      a -= p only if c_out > 0 (c_out: occurrences in the output);
  *   4. T == 0 (or < 0): greedy == top_k 1 with no scaling; else z = a * (1/T) in fp32;
  *   5. sort all ids by (order-preserving key of z descending, id ascending);
- *   6. top-k: keep the first min(k, #finite);  7. min-p: keep z - zmax >= ln(min_p);
+ *   6. top-k: keep the first min(k, #finite) -- or, in the keep-ties mode, every score not below
+ *      the k-th largest (what masking "logits < k-th value" gives);
+ *   7. min-p: keep z - zmax >= ln(min_p);
  *   8. top-p: smallest prefix whose mass >= top_p * (mass of the survivors);
  *   9. softmax over the survivors in fp64 -> log-probabilities;
  *  10. exponential race: Philox4x32-10 word per token -> E ~ Exp(1);
@@ -211,7 +213,7 @@ static int row_scores_and_order(const void *logits, int32_t dtype, int64_t row_p
  */
 static void row_cut_and_draw(const float *z, const sort_item_t *order, int32_t V, int greedy,
                              const row_params_t *rp, uint32_t R, uint64_t step,
-                             const float *exp1_row /* NULL: Philox */,
+                             const float *exp1_row /* NULL: Philox */, int keep_ties,
                              double ln_min_p_shift, double top_p_shift,
                              albireo_oracle_row_t *out, double *e /* scratch [V] */)
 {
@@ -225,7 +227,12 @@ static void row_cut_and_draw(const float *z, const sort_item_t *order, int32_t V
 
     /* 6. top-k */
     int32_t L = n_fin;
-    if (top_k >= 1 && top_k < V && top_k < L) L = top_k;
+    if (top_k >= 1 && top_k < V && top_k < L) {
+        L = top_k;
+        /* keep-ties mode: everything equal to the k-th largest score stays (equal scores have equal keys) */
+        if (keep_ties && !greedy)
+            while (L < n_fin && order[L].key == order[L - 1].key) ++L;
+    }
     if (L < 1) L = 1;
     out->n_fin = n_fin;
     out->n_topk = L;
@@ -322,6 +329,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                           const uint64_t *seeds, uint64_t step, uint32_t row_base,
                           const float *exp1 /* [B, V] Exp(1) variates, or NULL */,
                           const int32_t *out_start /* [B] where the output begins in each history, or NULL: 0 */,
+                          uint32_t flags /* bit 1 (value 2): top-k keeps ties */,
                           int32_t row_begin, int32_t row_end,
                           albireo_oracle_row_t *rows_out,
                           int32_t topk_cap, int32_t *topk_ids,
@@ -345,7 +353,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                                           out_start ? out_start[b] : 0, &rp, counts, z, order);
         albireo_oracle_row_t *o = &rows_out[b];
         row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step,
-                         exp1 ? exp1 + (int64_t)b * V : NULL, 0.0, 0.0, o, e);
+                         exp1 ? exp1 + (int64_t)b * V : NULL, (flags & 2u) != 0, 0.0, 0.0, o, e);
 
         if (topk_ids) for (int32_t j = 0; j < topk_cap; ++j)
             topk_ids[(int64_t)b * topk_cap + j] = (j < o->n_topk) ? order[j].id : -1;
@@ -380,7 +388,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
                                const float *min_p, const float *rep, const float *pres, const float *freq,
                                const int32_t *hist_ids, const int32_t *hist_off,
                                const uint64_t *seeds, uint64_t step, uint32_t row_base,
-                               const float *exp1, const int32_t *out_start,
+                               const float *exp1, const int32_t *out_start, uint32_t flags,
                                int32_t b, double ln_min_p_shift, double top_p_shift,
                                albireo_oracle_row_t *row_out, int32_t *sorted_ids, float *sorted_z,
                                double *sorted_g)
@@ -398,7 +406,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
     int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl,
                                       out_start ? out_start[b] : 0, &rp, counts, z, order);
     const float *exp1_row = exp1 ? exp1 + (int64_t)b * V : NULL;
-    row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, exp1_row,
+    row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, exp1_row, (flags & 2u) != 0,
                      ln_min_p_shift, top_p_shift, row_out, e);
     const double zmax = (double)z[order[0].id];
     for (int32_t j = 0; j < V; ++j) {

@@ -923,6 +923,14 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         bool clobbered = false;
         if (find_ok) C1 = resolve_cut<DT>(s, h, c, zmax, bin, false, n_topk, cb, Cfin, clobbered);
         if (clobbered) have_hist = have_mass = false;
+        if (a.flags & ALBIREO_FLAG_TOPK_KEEP_TIES) {
+            // every id of the k-th largest key stays; how many that makes takes a count over the row
+            C1 &= 0xFFFFFFFF00000000ull;
+            const uint32_t k1 = (uint32_t)(C1 >> 32);
+            uint32_t local = 0;
+            for_each_score<DT>(c, [&](int, float z) { const uint32_t kk = key_of(z); local += (kk >= k1 && kk < KEY_POS_INF); });
+            n_topk = block_sum_u64(s, local);
+        }
         if (want_topp && !have_mass) build_hist(false, true);
     }
     out.n_topk = (int32_t)n_topk;
@@ -952,7 +960,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         } else {
             u64 lm = 0;
             const uint32_t k1 = (uint32_t)(C1 >> 32); const int id1 = comp_idx(C1);
-            for_each_score<DT>(c, [&](int i, float z) { const uint32_t k = key_of(z); if (k > k1 || (k == k1 && i <= id1)) lm += mass_gen(__fsub_rn(z, zmax)); });
+            for_each_score<DT>(c, [&](int i, float z) { const uint32_t k = key_of(z); if (k > k1 || (k == k1 && (uint32_t)i <= (uint32_t)id1)) lm += mass_gen(__fsub_rn(z, zmax)); });
             Sp = block_sum_u64(s, lm);
         }
         double t = ceil((double)rp.top_p * (double)Sp);
@@ -995,7 +1003,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     };
     auto see = [&](int i, float z, bool may_queue) {
         const uint32_t k = key_of(z);
-        if (k > k2 || (k == k2 && i <= id2)) {
+        if (k > k2 || (k == k2 && (uint32_t)i <= (uint32_t)id2)) {
             const float d = __fsub_rn(z, zmax);
             S_local += mass_gen(d);
             n_local += 1;
@@ -1750,8 +1758,11 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
 
     const uint32_t kmax = s.runmax;    // the row's largest score is always a candidate
     bool topk_exact_known = true;      // is min(k, #finite) known without counting?
+    // keep-ties mode: the top-k stage keeps every score not below the k-th largest, i.e. exactly the
+    // candidates that are left once the list is cut at the k-th largest key
+    const bool keep_ties = has_topk && !rp.greedy && (a.flags & ALBIREO_FLAG_TOPK_KEEP_TIES);
     if (has_topk) {
-        if (n > SORT_MAX || n > 2 * k + 96) {
+        if (n > SORT_MAX || n > 2 * k + 96 || (keep_ties && n > k)) {
             uint32_t t = cand_select_exact(s, cs, n, k, tau_key, kmax);
             n = cand_compact(s, cs, n, t);
         }
@@ -1762,7 +1773,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     }
     if (n > SORT_MAX || n < 1) return false;
 
-    const int L6 = has_topk ? (n < k ? n : k) : n;
+    const int L6 = has_topk ? ((n < k || keep_ties) ? n : k) : n;
     int n_topk = L6;
     if (!topk_exact_known && a.out_num_topk) {
         // diagnostic only: count the finite scores of the row

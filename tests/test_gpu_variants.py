@@ -307,3 +307,29 @@ def test_split_history_full_vocabulary_and_limits(binding, sampler):
     w3.output_start = np.diff(w3.history_offsets).astype(np.int32)
     d, e = run(binding, sampler, w2), run(binding, sampler, w3)
     assert (d["tokens"] == e["tokens"]).all() and (d["logprobs"] == e["logprobs"]).all()
+
+
+# ------------------------------------------------------------------ top-k that keeps ties
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16, W.F16])
+@pytest.mark.parametrize("general", [0, 1], ids=["auto", "general"])
+def test_topk_keep_ties(binding, sampler, dtype, general):
+    base = W.random_small(701, B=48, V=9001, dtype=W.F32 if dtype == W.F16 else dtype, quantise=0.5)   # ties at every cut
+    w = W.as_f16(base) if dtype == W.F16 else base
+    w.topk_keep_ties = True
+    w.num_top = 6
+    flags = binding.FLAG_TOPK_KEEP_TIES | (binding.FLAG_FORCE_GENERAL if general else 0)
+    g, ref = check(binding, sampler, w, flags=flags)
+    strict = O.sample(W.random_small(701, B=48, V=9001, dtype=W.F32 if dtype == W.F16 else dtype, quantise=0.5))
+    assert (ref.rows["n_topk"] > strict.rows["n_topk"]).sum() >= 5          # the mode matters on these rows
+    assert (g["num_topk"] == ref.rows["n_topk"]).all()
+
+
+def test_topk_keep_ties_thousands_of_ties(binding, sampler):
+    rng = np.random.default_rng(71)
+    x = np.round(rng.standard_normal((6, 30000)) * 2).astype(np.float32)    # ~6000 elements per distinct value
+    w = W.Workload("ties", 6, 30000, W.BF16, W.f32_to_bf16_bits(x), temperature=np.full(6, 0.9, np.float32),
+                   top_k=np.array([1, 5, 50, 300, 2000, 29999], np.int32), top_p=np.full(6, 0.95, np.float32),
+                   seeds=np.arange(6, dtype=np.uint64), topk_keep_ties=True)
+    g, ref = check(binding, sampler, w, flags=binding.FLAG_TOPK_KEEP_TIES)
+    assert (g["num_topk"] == ref.rows["n_topk"]).all() and ref.rows["n_topk"][4] > 2500

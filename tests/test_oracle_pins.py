@@ -586,3 +586,44 @@ def test_split_history_through_the_batch_entry():
     w0 = W.random_small(53, B=12, V=300, dtype=W.F32)
     base = O.sample(w0)
     assert (base.tokens != got.tokens).any() or (base.logprobs != got.logprobs).any()
+
+
+# ------------------------------------------------------------------ top-k that keeps ties
+
+def test_topk_keep_ties_equals_masking_below_the_kth_value():
+    """Keep-ties top-k is what masking every logit below the k-th largest value gives (brute force
+    with numpy on quantised rows), and equals the strict top-k whenever the k-th value is unique."""
+    rng = np.random.default_rng(61)
+    for V in (7, 40, 300):
+        for trial in range(5):
+            x = (np.round(rng.standard_normal(V) * 1.5) * 0.5).astype(np.float32)      # many exact ties
+            x = x + np.float32(0.0)                 # no -0.0: the order puts it below +0.0, numpy's >= does not
+            for k in (1, 2, 3, V // 2, V - 1):
+                if k < 1:
+                    continue
+                w = one_row(x, T=1.0, top_k=k)
+                w.topk_keep_ties = True
+                o = O.sample(w, topk_cap=V, kept_cap=V)
+                kth = np.sort(x)[::-1][k - 1]
+                want = sorted(np.nonzero(x >= kth)[0].tolist())
+                got = sorted(i for i in o.topk_ids[0].tolist() if i >= 0)
+                assert got == want and o.rows["n_topk"][0] == len(want)
+                # the distribution over the kept set is the softmax of the masked row
+                masked = np.where(x >= kth, x.astype(np.float64), -np.inf)
+                lp = masked - scipy.special.logsumexp(masked)
+                assert abs(o.logprobs[0] - lp[o.tokens[0]]) < 1e-12
+                strict = O.sample(one_row(x, T=1.0, top_k=k), topk_cap=V)
+                if (x >= kth).sum() == k:          # no tie reaches beyond the k-th place: same set as the strict cut
+                    assert (strict.topk_ids == o.topk_ids).all() and strict.tokens[0] == o.tokens[0]
+                else:
+                    assert strict.rows["n_topk"][0] == k < o.rows["n_topk"][0]
+
+
+def test_topk_keep_ties_leaves_greedy_and_other_cuts_alone():
+    x = np.array([[2.0, 2.0, 1.0, 2.0, 0.5, 1.0]], dtype=np.float32)
+    g = one_row(x, T=0.0, top_k=2); g.topk_keep_ties = True
+    assert O.sample(g).tokens[0] == 0 and O.sample(g).rows["n_keep"][0] == 1       # greedy: lowest id of the maxima
+    w = one_row(x, T=1.0, top_k=2, top_p=0.5); w.topk_keep_ties = True
+    o = O.sample(w, kept_cap=6)
+    assert o.rows["n_topk"][0] == 3                                                 # the three 2.0s
+    assert [i for i in o.kept_ids[0] if i >= 0] == [0, 1]                           # top-p on their mass: 1/3 + 1/3 >= 0.5
