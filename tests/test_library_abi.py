@@ -77,3 +77,31 @@ def test_product_does_not_import_the_oracle():
             if fn.endswith((".py", ".cu", ".cuh", ".h", ".cpp")):
                 src = open(os.path.join(dirpath, fn)).read()
                 assert "oracle" not in src.lower() or fn == "workloads.py", fn
+
+
+def test_binding_struct_and_constants_match_the_header(tmp_path):
+    """The ctypes mirror of albireo_sample_ext_t has the C layout (size and every field offset), and the
+    binding's constants are the header's: checked by compiling the header with the host C compiler."""
+    import subprocess
+    from paper_2606_01927_b200 import binding
+    fields = [f[0] for f in binding.SampleExt._fields_]
+    prog = ['#include <stdio.h>', '#include <stddef.h>', '#include "albireo_sample.h"', 'int main(void) {',
+            '  printf("sizeof %zu\\n", sizeof(albireo_sample_ext_t));']
+    prog += [f'  printf("{f} %zu\\n", offsetof(albireo_sample_ext_t, {f}));' for f in fields]
+    for name in ("ALBIREO_F32", "ALBIREO_BF16", "ALBIREO_F16", "ALBIREO_MAX_VOCAB", "ALBIREO_MAX_NUM_TOP",
+                 "ALBIREO_FLAG_FORCE_GENERAL", "ALBIREO_FLAG_TOPK_KEEP_TIES", "ALBIREO_FIXED_MAX_HISTORY", "ALBIREO_OK"):
+        prog.append(f'  printf("{name} %lld\\n", (long long){name});')
+    prog += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(prog))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = dict(line.split() for line in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    assert int(out["sizeof"]) == C.sizeof(binding.SampleExt)
+    for f in fields:
+        assert int(out[f]) == getattr(binding.SampleExt, f).offset, f
+    assert (int(out["ALBIREO_F32"]), int(out["ALBIREO_BF16"]), int(out["ALBIREO_F16"])) == (binding.F32, binding.BF16, binding.F16)
+    assert int(out["ALBIREO_MAX_VOCAB"]) == binding.MAX_VOCAB and int(out["ALBIREO_MAX_NUM_TOP"]) == binding.MAX_NUM_TOP
+    assert int(out["ALBIREO_FLAG_FORCE_GENERAL"]) == binding.FLAG_FORCE_GENERAL
+    assert int(out["ALBIREO_FLAG_TOPK_KEEP_TIES"]) == binding.FLAG_TOPK_KEEP_TIES
+    assert int(out["ALBIREO_FIXED_MAX_HISTORY"]) == binding.FIXED_MAX_HISTORY and int(out["ALBIREO_OK"]) == binding.OK
