@@ -57,6 +57,7 @@ struct SampleArgs {
     int64_t row_stride;
     int32_t nseg;               // pieces per row (1: rows are contiguous)
     int64_t seg_stride;         // elements between consecutive pieces of a row
+    int32_t Vs, vps;            // elements and 16-byte vectors per piece (worked out on the host: no division on the device)
     const float *temperature;
     const int32_t *top_k;
     const float *top_p, *min_p, *rep, *pres, *freq;
@@ -1127,6 +1128,7 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
 }
 // copies vectors [v0, v0 + nv) of the row to dst, piece by piece; the bytes were announced to `bar`
 __device__ __forceinline__ void ring_copy(const Ring &rg, void *dst, const uint4 *vp, int v0, int nv, uint64_t *bar) {
+    if (rg.vps == 0x7FFFFFFF) { bulk_g2s(dst, vp + v0, (uint32_t)nv * 16u, bar); return; }    // one piece
     unsigned char *d = (unsigned char *)dst;
     int j = v0 / rg.vps, off = v0 - j * rg.vps;
     while (nv > 0) {
@@ -1472,9 +1474,7 @@ __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c
     const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
     const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
     {
-        s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
-        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
-        for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
+        // the copies first: every cycle before them is a cycle nothing is on its way
         for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
         mbar_init(&rg.bar[MAX_STAGES - 1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1483,6 +1483,9 @@ __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c
         const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
         for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
         s.issued = (uint32_t)npre;
+        s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
+        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
+        for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
     }
 }
 
@@ -1800,32 +1803,32 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     const int b = blockIdx.x;
     const int V = a.V;
 
-    HistBins h;
-    h.cnt = (uint32_t *)smem;
-    h.limb = (uint32_t *)(smem + HIST_BINS * 4);
-    h.list = (u64 *)(smem + HIST_BINS * 16);
-    h.acc = h.list + GL_CAP;
     Ring rg;
     rg.nstages = a.nstages;
-    rg.vps = a.nseg > 1 ? (V / a.nseg) / Elem<DT>::PER_VEC : 0x7FFFFFFF;
+    rg.vps = a.vps;
     rg.seg_vecs = a.seg_stride * Elem<DT>::SIZE / 16;
     rg.buf = smem + COMMON_BYTES;
     rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
-    HistSmem hs;
-    const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
-    hs.bitmap = (uint32_t *)((unsigned char *)rg.bar + MAX_STAGES * 8);
-    hs.coarse = hs.bitmap + (nwords + 1);
-    hs.counts = hs.coarse + (ncoarse + 1);
-
     RowCtx c;
     c.row = (const char *)a.logits + (size_t)b * (size_t)a.row_stride * Elem<DT>::SIZE;
     c.V = V;
-    c.nseg = a.nseg; c.Vs = V / a.nseg; c.seg_bytes = a.seg_stride * Elem<DT>::SIZE;
+    c.nseg = a.nseg; c.Vs = a.Vs; c.seg_bytes = a.seg_stride * Elem<DT>::SIZE;
     // The ring is started before anything else is read, the row's own parameters included: their
     // loads and the first tiles then travel together.  A row that turns out to need the general
     // path waits for these copies before it reuses the shared memory.
     const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
     if (ring_started) candidate_begin<DT>(s, rg, c);
+
+    HistBins h;
+    h.cnt = (uint32_t *)smem;
+    h.limb = (uint32_t *)(smem + HIST_BINS * 4);
+    h.list = (u64 *)(smem + HIST_BINS * 16);
+    h.acc = h.list + GL_CAP;
+    HistSmem hs;
+    const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
+    hs.bitmap = (uint32_t *)((unsigned char *)rg.bar + MAX_STAGES * 8);
+    hs.coarse = hs.bitmap + (nwords + 1);
+    hs.counts = hs.coarse + (ncoarse + 1);
 
     RowParams rp;
     rp.T = a.temperature ? a.temperature[b] : 1.0f;
@@ -1960,6 +1963,7 @@ int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, cons
             *why = "rows in pieces need 16-byte aligned pieces, row stride, segment stride and base"; return ALBIREO_EUNSUPPORTED;
         }
         a.nseg = (int32_t)t; a.seg_stride = ext->segment_stride_elems;
+        a.Vs = (int32_t)Vs; a.vps = (int32_t)(Vs * esz / 16);
     } else if (ext->num_segments < 0) { *why = "num_segments is negative"; return ALBIREO_EINVAL; }
     a.out_start = ext->history_output_start;
     if (ext->exp1) {
@@ -2094,7 +2098,7 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
 
     SampleArgs a;
     memset(&a, 0, sizeof a);
-    a.logits = logits; a.B = B; a.V = V; a.row_stride = V; a.nseg = 1; a.elem_size = (int32_t)esize;
+    a.logits = logits; a.B = B; a.V = V; a.row_stride = V; a.nseg = 1; a.Vs = V; a.vps = 0x7FFFFFFF; a.elem_size = (int32_t)esize;
     a.temperature = temperature; a.top_k = top_k; a.top_p = top_p; a.min_p = min_p;
     a.rep = repetition_penalty; a.pres = presence_penalty; a.freq = frequency_penalty;
     a.hist_ids = history_ids; a.hist_off = history_offsets;
@@ -2290,7 +2294,7 @@ extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32
 
     SampleArgs a;
     memset(&a, 0, sizeof a);
-    a.logits = logits; a.B = B; a.V = V; a.row_stride = V; a.nseg = 1; a.elem_size = (int32_t)esize;
+    a.logits = logits; a.B = B; a.V = V; a.row_stride = V; a.nseg = 1; a.Vs = V; a.vps = 0x7FFFFFFF; a.elem_size = (int32_t)esize;
     a.temperature = temperature; a.top_k = top_k; a.top_p = top_p; a.min_p = min_p;
     a.rep = repetition_penalty; a.pres = presence_penalty; a.freq = frequency_penalty;
     a.hist_ids = history_ids; a.hist_off = history_offsets;
