@@ -228,9 +228,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch each step from Python instead of one CUDA graph")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--general-path", action="store_true", help="force every row down the general path")
-    ap.add_argument("--variant", default="none", choices=["none", "f16", "exp1", "feedback"],
+    ap.add_argument("--variant", default="none", choices=["none", "f16", "exp1", "feedback", "fullvocab"],
                     help="the same workload as binary16 logits, with a pre-generated Exp(1) table, or with the "
-                         "early-feedback targets (next input ids + pinned host ring)")
+                         "early-feedback targets (next input ids + pinned host ring), or with log-probabilities "
+                         "relative to the full vocabulary")
     ap.add_argument("--sequence-parallel", default=None, choices=["a2a", "gather"],
                     help="secondary mode: logits start as per-rank vocabulary shards; time all-to-all + sample + "
                          "gather (a2a) or the gather-to-one-rank arrangement it replaces (gather)")
@@ -289,6 +290,8 @@ def main():
     out_tok = torch.empty(w.B, dtype=torch.int32, device=dev)
     out_lp = torch.empty(w.B, dtype=torch.float32, device=dev)
     flags = binding.FLAG_FORCE_GENERAL if args.general_path else 0
+    if args.variant == "fullvocab":
+        flags |= binding.FLAG_LOGPROB_FULL_VOCAB
     stream = torch.cuda.Stream(device=dev)
     if args.variant == "feedback":
         t["backfill_ids"] = torch.zeros(w.backfill_len, dtype=torch.int32, device=dev)

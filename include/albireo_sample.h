@@ -69,6 +69,11 @@ enum {
                                          (what masking "logits < k-th value" gives) instead of
                                          exactly k ids; equal means equal in the order, so -0.0
                                          stays below +0.0; greedy rows are not affected          */
+#define ALBIREO_FLAG_LOGPROB_FULL_VOCAB 4u /* out_logprobs and out_top_logprobs are relative to the
+                                         softmax over every finite score of the row (after penalties
+                                         and temperature; greedy rows: over the unscaled scores)
+                                         instead of the final kept set; the token drawn does not
+                                         change.  Costs one more pass over the row, from L2        */
 
 /*
  * Optional arguments of albireo_sample (pass NULL for all defaults).  Zero-initialise,

@@ -56,7 +56,8 @@ typedef struct {
     int32_t greedy;       /* 1 if the row was treated as greedy                 */
     double logprob;       /* log-probability of `token` in the final kept set   */
     double z_max;         /* largest z (as double)                              */
-    double S;             /* sum of exp(z - zmax) over the final kept set       */
+    double S;             /* normaliser of the log-probabilities: sum of exp(z - zmax) over the final
+                             kept set (over all finite scores in the full-vocabulary mode)      */
     double race_gap;      /* best - second best race score (+inf if n_keep==1)  */
     double minp_margin;   /* min_j |d_j - ln(min_p)| over the step-6 set (+inf if off) */
     double topp_margin;   /* distance of top_p*S' to the nearest cumulative sum, / S' (+inf if off) */
@@ -213,7 +214,7 @@ static int row_scores_and_order(const void *logits, int32_t dtype, int64_t row_p
  */
 static void row_cut_and_draw(const float *z, const sort_item_t *order, int32_t V, int greedy,
                              const row_params_t *rp, uint32_t R, uint64_t step,
-                             const float *exp1_row /* NULL: Philox */, int keep_ties,
+                             const float *exp1_row /* NULL: Philox */, int keep_ties, int full_vocab,
                              double ln_min_p_shift, double top_p_shift,
                              albireo_oracle_row_t *out, double *e /* scratch [V] */)
 {
@@ -272,9 +273,17 @@ static void row_cut_and_draw(const float *z, const sort_item_t *order, int32_t V
     }
     out->n_keep = L;
 
-    /* 9. softmax over the final kept set */
+    /* 9. softmax over the final kept set -- or, in the full-vocabulary mode, over every finite score of
+          the row (the cuts then decide what may be drawn, not what the probabilities are relative to) */
     double S = 0.0;
-    for (int32_t j = 0; j < L; ++j) S += e[j];
+    if (full_vocab) {
+        for (int32_t j = 0; j < V; ++j) {
+            double zj = (double)z[order[j].id];
+            if (isfinite(zj)) S += exp(zj - zmax);
+        }
+    } else {
+        for (int32_t j = 0; j < L; ++j) S += e[j];
+    }
     out->S = S;
     out->z_max = zmax;
     const double lnS = log(S);
@@ -329,7 +338,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                           const uint64_t *seeds, uint64_t step, uint32_t row_base,
                           const float *exp1 /* [B, V] Exp(1) variates, or NULL */,
                           const int32_t *out_start /* [B] where the output begins in each history, or NULL: 0 */,
-                          uint32_t flags /* bit 1 (value 2): top-k keeps ties */,
+                          uint32_t flags /* value 2: top-k keeps ties; value 4: log-probabilities relative to the full vocabulary */,
                           int32_t row_begin, int32_t row_end,
                           albireo_oracle_row_t *rows_out,
                           int32_t topk_cap, int32_t *topk_ids,
@@ -353,7 +362,7 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
                                           out_start ? out_start[b] : 0, &rp, counts, z, order);
         albireo_oracle_row_t *o = &rows_out[b];
         row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step,
-                         exp1 ? exp1 + (int64_t)b * V : NULL, (flags & 2u) != 0, 0.0, 0.0, o, e);
+                         exp1 ? exp1 + (int64_t)b * V : NULL, (flags & 2u) != 0, (flags & 4u) != 0, 0.0, 0.0, o, e);
 
         if (topk_ids) for (int32_t j = 0; j < topk_cap; ++j)
             topk_ids[(int64_t)b * topk_cap + j] = (j < o->n_topk) ? order[j].id : -1;
@@ -406,7 +415,7 @@ int albireo_oracle_row_shifted(const void *logits, int32_t B, int32_t V, int32_t
     int greedy = row_scores_and_order(logits, dtype, (int64_t)b * row_stride, V, h, hl,
                                       out_start ? out_start[b] : 0, &rp, counts, z, order);
     const float *exp1_row = exp1 ? exp1 + (int64_t)b * V : NULL;
-    row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, exp1_row, (flags & 2u) != 0,
+    row_cut_and_draw(z, order, V, greedy, &rp, row_base + (uint32_t)b, step, exp1_row, (flags & 2u) != 0, (flags & 4u) != 0,
                      ln_min_p_shift, top_p_shift, row_out, e);
     const double zmax = (double)z[order[0].id];
     for (int32_t j = 0; j < V; ++j) {

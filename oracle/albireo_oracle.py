@@ -95,7 +95,7 @@ def _common_args(w):
         _ptr(w.seeds, np.uint64), C.c_uint64(w.step), C.c_uint32(w.row_base),
         _ptr(getattr(w, "exp1", None), np.float32),
         _ptr(getattr(w, "output_start", None), np.int32),
-        C.c_uint32(2 if getattr(w, "topk_keep_ties", False) else 0),
+        C.c_uint32((2 if getattr(w, "topk_keep_ties", False) else 0) | (4 if getattr(w, "logprob_full_vocab", False) else 0)),
     ]
 
 

@@ -705,6 +705,51 @@ __device__ __forceinline__ u64 mass_gen(float d) {
     return d < -28.5f ? 0ull : __float2ull_rn(__expf(d) * FX_SCALE);
 }
 
+// Mass of the whole row, sum of exp(z - zmax) over its finite scores in 2^40 fixed point: the
+// normaliser of the log-probabilities in the full-vocabulary mode.  One more pass over the row (it
+// was just read, so mostly from L2), four loads in flight; vectors with nothing within 29 of the
+// maximum carry no mass and are skipped by the packed test of the candidate path; the masses of a
+// vector are added in fp32 (a fixed order) and turned into fixed point once.  The same in every thread.
+template <int DT>
+__device__ u64 full_vocab_mass(BlockScratch &s, const RowCtx &c, float zmax) {
+    typedef Elem<DT> E;
+    typedef VecTest<DT> T;
+    const int V = c.V;
+    const uintptr_t addr = (uintptr_t)c.row;
+    int head = (int)(((16u - (uint32_t)(addr & 15u)) & 15u) / E::SIZE);
+    if (head > V) head = V;
+    const int nvec = (V - head) / E::PER_VEC;
+    const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
+    const uint32_t thr = T::raw_threshold(key_of(zmax - 29.0f), c.invT);
+    u64 local = 0;
+    for (int v0 = threadIdx.x; v0 < nvec; v0 += 4 * NT) {
+        uint4 q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) q[u] = (v0 + u * NT < nvec) ? __ldg(vec_ptr<DT>(c, vp, v0 + u * NT)) : T::fill();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int v = v0 + u * NT;
+            if (v >= nvec) break;
+            if (!T::may_pass(q[u], thr, c.invT)) continue;
+            const int i0 = head + v * E::PER_VEC;
+            uint32_t m = 0;
+            if (c.has_hist) m = __funnelshift_r(c.bitmap[i0 >> 5], c.bitmap[(i0 >> 5) + 1], i0 & 31);
+            float acc = 0.0f;
+#pragma unroll
+            for (int e = 0; e < E::PER_VEC; ++e) {
+                const float d = __fsub_rn(__fmul_rn(E::get(q[u], e), c.invT), zmax);
+                if (!((m >> e) & 1u) && d >= -28.5f) acc += __expf(d);
+            }
+            local += __float2ull_rn(acc * FX_SCALE);
+        }
+    }
+    for_each_score_rest<DT>(c, head, nvec, [&](int, float z) {
+        const float d = __fsub_rn(z, zmax);
+        if (d > -3.0e38f) local += mass_gen(d);         // -inf (and NaN) carry no mass
+    });
+    return block_sum_u64(s, local);
+}
+
 // value-linear bin of a finite score z <= zmax; monotone: a larger z never gets a larger bin
 __device__ __forceinline__ int bin_of(float z, float zmax) {
     int b = __float2int_rz(__fsub_rn(zmax, z) * BIN_SCALE);
@@ -881,12 +926,14 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         return (int)~(uint32_t)block_max_u64(s, best);
     };
 
+    const bool full_lp = (a.flags & ALBIREO_FLAG_LOGPROB_FULL_VOCAB) != 0;
     if (rp.greedy || n_fin <= 1) {
         out.token = top_id(); out.logprob = 0.0f; out.n_keep = 1; out.n_topk = 1;
+        if (full_lp) out.logprob = (float)-(log((double)full_vocab_mass<DT>(s, c, zmax)) - LN2_40);
         if (a.dbg_topk_ids && a.dbg_cap >= 1 && threadIdx.x == 0) a.dbg_topk_ids[(int64_t)b * a.dbg_cap] = out.token;
         if (a.num_top > 0 && threadIdx.x == 0) {
             a.out_top_ids[(int64_t)b * a.num_top] = out.token;
-            a.out_top_logprobs[(int64_t)b * a.num_top] = 0.0f;
+            a.out_top_logprobs[(int64_t)b * a.num_top] = out.logprob;
         }
         return;
     }
@@ -1053,10 +1100,10 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     const u64 n_keep = block_sum_u64(s, n_local);
     const u64 G = block_max_u64(s, g_best);
     const int tok = comp_idx(G);
-    const double lnS = log((double)S_fx) - LN2_40;
+    const double lnS = log((double)(full_lp ? full_vocab_mass<DT>(s, c, zmax) : S_fx)) - LN2_40;
     float z_tok = score_of(c, tok, Elem<DT>::load(elem_ptr<DT>(c, tok), 0));
     out.token = tok;                                   // (a single kept element wins its own race)
-    out.logprob = (n_keep == 1) ? 0.0f : (float)(((double)z_tok - (double)zmax) - lnS);
+    out.logprob = (n_keep == 1 && !full_lp) ? 0.0f : (float)(((double)z_tok - (double)zmax) - lnS);
     out.n_keep = (int32_t)n_keep;
 
     if (want_top_list) {
@@ -1080,7 +1127,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
             if (rank < a.num_top) {
                 const int64_t o = (int64_t)b * a.num_top + rank;
                 a.out_top_ids[o] = comp_idx(C);
-                a.out_top_logprobs[o] = (n_keep == 1) ? 0.0f : (float)(((double)unkey((uint32_t)(C >> 32)) - (double)zmax) - lnS);
+                a.out_top_logprobs[o] = (n_keep == 1 && !full_lp) ? 0.0f : (float)(((double)unkey((uint32_t)(C >> 32)) - (double)zmax) - lnS);
             }
         }
         __syncthreads();
@@ -1319,8 +1366,9 @@ __device__ __forceinline__ void cand_append_one(BlockScratch &s, const CandSmem 
 // score is zmax.  Step 1 (all threads): each candidate's rank by counting (several threads share
 // the comparisons of one candidate when n is small), its mass and its race score, written to its
 // sorted position.  Step 2 (warp 0): the cuts as prefix operations and the argmax of the race.
+// `full_fx` != 0: the log-probabilities are relative to that mass (the whole row's) instead of the kept set's.
 __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, float zmax, bool has_minp,
-                            const RowParams &rp, const SampleArgs &a, int b, RowOut &out) {
+                            const RowParams &rp, const SampleArgs &a, int b, RowOut &out, u64 full_fx) {
     const int lane = threadIdx.x & 31;
     // `parts` threads share one candidate's comparisons; the threads after them (from the next warp
     // boundary on) take one candidate each for the race term and the mass, so those long dependent
@@ -1393,9 +1441,9 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         L8 = __reduce_add_sync(0xFFFFFFFFu, cnt);
         S_fx = __shfl_sync(0xFFFFFFFFu, last, (L8 - 1) / per);
     }
-    const float lnS = logf((float)S_fx * (1.0f / FX_SCALE));
+    const float lnS = logf((float)(full_fx ? full_fx : S_fx) * (1.0f / FX_SCALE));
     int tok = comp_idx(sorted[0]);
-    float lp_tok = 0.0f;
+    float lp_tok = full_fx ? __fsub_rn(unkey((uint32_t)(sorted[0] >> 32)), zmax) - lnS : 0.0f;
     if (L8 > 1) {
         // argmax of the race score over the kept prefix (ties: lowest id, via the low word ~id)
         u64 best = 0; int bestq = 0;
@@ -1412,7 +1460,7 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         for (int q = lane; q < a.num_top && q < L8; q += 32) {
             const int64_t o = (int64_t)b * a.num_top + q;
             a.out_top_ids[o] = comp_idx(sorted[q]);
-            a.out_top_logprobs[o] = (L8 == 1) ? 0.0f : __fsub_rn(unkey((uint32_t)(sorted[q] >> 32)), zmax) - lnS;
+            a.out_top_logprobs[o] = (L8 == 1 && !full_fx) ? 0.0f : __fsub_rn(unkey((uint32_t)(sorted[q] >> 32)), zmax) - lnS;
         }
     }
 }
@@ -1786,7 +1834,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         n_topk = has_topk ? (int)(nfin < (u64)k ? nfin : (u64)k) : (int)nfin;
     }
     out.n_topk = n_topk;
-    final_stage(s, cs, n, L6, unkey(kmax), has_minp, rp, a, b, out);
+    const u64 full_fx = (a.flags & ALBIREO_FLAG_LOGPROB_FULL_VOCAB) ? full_vocab_mass<DT>(s, c, unkey(kmax)) : 0ull;
+    final_stage(s, cs, n, L6, unkey(kmax), has_minp, rp, a, b, out, full_fx);
     return true;
 }
 

@@ -54,7 +54,8 @@ class Workload:
     (early feedback, §5.2).  ``output_start`` (int32 ``[B]``) splits each history into prompt
     (the first ``output_start[b]`` ids) and generated output (the rest): the repetition penalty then
     looks at both, the presence and frequency penalties at the output alone.
-    ``topk_keep_ties`` switches top-k to "keep every score not below the k-th largest".
+    ``topk_keep_ties`` switches top-k to "keep every score not below the k-th largest";
+    ``logprob_full_vocab`` reports log-probabilities relative to the softmax over the whole row.
     """
 
     name: str
@@ -80,6 +81,7 @@ class Workload:
     backfill_len: int = 0
     output_start: Optional[np.ndarray] = None
     topk_keep_ties: bool = False
+    logprob_full_vocab: bool = False
     notes: dict = field(default_factory=dict)
 
     @property
@@ -121,7 +123,8 @@ class Workload:
             history_ids=hid, history_offsets=hoff, seeds=cut(self.seeds), step=self.step,
             row_base=self.row_base + lo, num_top=self.num_top, exp1=cut(self.exp1),
             backfill_index=cut(self.backfill_index), backfill_len=self.backfill_len,
-            output_start=cut(self.output_start), topk_keep_ties=self.topk_keep_ties, notes=dict(self.notes))
+            output_start=cut(self.output_start), topk_keep_ties=self.topk_keep_ties,
+            logprob_full_vocab=self.logprob_full_vocab, notes=dict(self.notes))
 
 
 # --------------------------------------------------------------------------- helpers

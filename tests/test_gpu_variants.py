@@ -333,3 +333,23 @@ def test_topk_keep_ties_thousands_of_ties(binding, sampler):
                    seeds=np.arange(6, dtype=np.uint64), topk_keep_ties=True)
     g, ref = check(binding, sampler, w, flags=binding.FLAG_TOPK_KEEP_TIES)
     assert (g["num_topk"] == ref.rows["n_topk"]).all() and ref.rows["n_topk"][4] > 2500
+
+
+# ------------------------------------------------------------------ log-probabilities relative to the full vocabulary
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+@pytest.mark.parametrize("general", [0, 1], ids=["auto", "general"])
+def test_full_vocabulary_logprobs(binding, sampler, dtype, general):
+    w = W.random_small(801, B=48, V=9001, dtype=dtype)
+    w.logprob_full_vocab = True
+    w.num_top = 5
+    flags = binding.FLAG_LOGPROB_FULL_VOCAB | (binding.FLAG_FORCE_GENERAL if general else 0)
+    g, ref = check(binding, sampler, w, flags=flags)
+    plain = O.sample(W.random_small(801, B=48, V=9001, dtype=dtype))
+    assert (plain.tokens == ref.tokens).all() and (ref.logprobs < plain.logprobs - 1e-9).sum() >= 20
+
+
+def test_full_vocabulary_logprobs_full_size_rows(binding, sampler):
+    w = W.config4(B=48)
+    w.logprob_full_vocab = True
+    check(binding, sampler, w, flags=binding.FLAG_LOGPROB_FULL_VOCAB)

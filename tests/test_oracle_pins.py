@@ -627,3 +627,32 @@ def test_topk_keep_ties_leaves_greedy_and_other_cuts_alone():
     o = O.sample(w, kept_cap=6)
     assert o.rows["n_topk"][0] == 3                                                 # the three 2.0s
     assert [i for i in o.kept_ids[0] if i >= 0] == [0, 1]                           # top-p on their mass: 1/3 + 1/3 >= 0.5
+
+
+# ------------------------------------------------------------------ log-probabilities relative to the full vocabulary
+
+def test_full_vocabulary_logprobs_equal_library_log_softmax_whatever_the_cuts():
+    rng = np.random.default_rng(67)
+    B, V = 10, 500
+    x = (rng.standard_normal((B, V)) * 2.5).astype(np.float32)
+    x[3, ::7] = -np.inf                                     # masked entries carry no mass
+    T = np.float32(0.8)
+    ref = scipy.special.log_softmax((x * (np.float32(1.0) / T)).astype(np.float64), axis=1)
+    base = O.sample(one_row(x, T=float(T), top_k=20, top_p=0.9, min_p=0.02, seed=4, num_top=6))
+    w = one_row(x, T=float(T), top_k=20, top_p=0.9, min_p=0.02, seed=4, num_top=6)
+    w.logprob_full_vocab = True
+    o = O.sample(w)
+    assert (o.tokens == base.tokens).all() and (o.rows["n_keep"] == base.rows["n_keep"]).all()   # the draw is untouched
+    for b in range(B):
+        assert abs(o.logprobs[b] - ref[b, o.tokens[b]]) < 1e-12
+        for j in range(6):
+            if o.top_ids[b, j] >= 0:
+                assert abs(o.top_logprobs[b, j] - ref[b, o.top_ids[b, j]]) < 1e-12
+        assert o.logprobs[b] <= base.logprobs[b] + 1e-15      # the kept set's normaliser is the smaller one
+    # greedy rows: the arg max under the softmax of the unscaled scores
+    g = one_row(x, T=0.0)
+    g.logprob_full_vocab = True
+    og = O.sample(g)
+    ref0 = scipy.special.log_softmax(x.astype(np.float64), axis=1)
+    for b in range(B):
+        assert og.tokens[b] == int(np.argmax(x[b])) and abs(og.logprobs[b] - ref0[b, og.tokens[b]]) < 1e-12
