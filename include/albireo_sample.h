@@ -73,7 +73,10 @@ enum {
                                          softmax over every finite score of the row (after penalties
                                          and temperature; greedy rows: over the unscaled scores)
                                          instead of the final kept set; the token drawn does not
-                                         change.  Costs one more pass over the row, from L2        */
+                                         change.  Costs one more pass over the row, from L2.  A
+                                         top-N list (num_top > 0) then holds the first entries of the
+                                         whole row's order, not of the kept set; rows with such a
+                                         list take the general path                               */
 
 /*
  * Optional arguments of albireo_sample (pass NULL for all defaults).  Zero-initialise,

@@ -370,9 +370,11 @@ int albireo_oracle_sample(const void *logits, int32_t B, int32_t V, int32_t dtyp
             kept_ids[(int64_t)b * kept_cap + j] = (j < o->n_keep) ? order[j].id : -1;
         if (top_ids && top_logprobs) {
             const double lnS = log(o->S);
+            /* the list runs over the final kept set; in the full-vocabulary mode over every finite score */
+            const int32_t list_len = (flags & 4u) ? o->n_fin : o->n_keep;
             for (int32_t j = 0; j < num_top; ++j) {
                 int64_t q = (int64_t)b * num_top + j;
-                if (j < o->n_keep) {
+                if (j < list_len) {
                     top_ids[q] = order[j].id;
                     top_logprobs[q] = ((double)z[order[j].id] - o->z_max) - lnS;
                 } else {

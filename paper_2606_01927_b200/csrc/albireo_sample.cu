@@ -170,6 +170,7 @@ struct BlockScratch {
     uint32_t done[MAX_STAGES];   // warps finished with each ring stage
     uint32_t maint_at;           // tile index before which every warp meets (0xFFFFFFFF: none)
     uint32_t issued;             // tiles whose copy has been issued so far
+    uint32_t nfin_cap;           // general path: min(#finite scores, ALBIREO_MAX_NUM_TOP + 1), parked here until the list is written
 };
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -927,21 +928,12 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     };
 
     const bool full_lp = (a.flags & ALBIREO_FLAG_LOGPROB_FULL_VOCAB) != 0;
-    if (rp.greedy || n_fin <= 1) {
-        out.token = top_id(); out.logprob = 0.0f; out.n_keep = 1; out.n_topk = 1;
-        if (full_lp) out.logprob = (float)-(log((double)full_vocab_mass<DT>(s, c, zmax)) - LN2_40);
-        if (a.dbg_topk_ids && a.dbg_cap >= 1 && threadIdx.x == 0) a.dbg_topk_ids[(int64_t)b * a.dbg_cap] = out.token;
-        if (a.num_top > 0 && threadIdx.x == 0) {
-            a.out_top_ids[(int64_t)b * a.num_top] = out.token;
-            a.out_top_logprobs[(int64_t)b * a.num_top] = out.logprob;
-        }
-        return;
-    }
-
+    if (threadIdx.x == 0) s.nfin_cap = (uint32_t)(n_fin < (u64)ALBIREO_MAX_NUM_TOP + 1 ? n_fin : (u64)ALBIREO_MAX_NUM_TOP + 1);
     const u64 Cfin = (u64)KEY_MIN_FINITE << 32;
-    const bool want_k = rp.top_k >= 1 && rp.top_k < V && (u64)rp.top_k < n_fin;
-    const bool want_minp = rp.min_p > 0.0f;
-    const bool want_topp = rp.top_p < 1.0f;
+    const int top_k = rp.greedy ? 1 : rp.top_k;          // (a greedy row gets here only for the whole-vocabulary list)
+    const bool want_k = top_k >= 1 && top_k < V && (u64)top_k < n_fin;
+    const bool want_minp = !rp.greedy && rp.min_p > 0.0f;
+    const bool want_topp = !rp.greedy && rp.top_p < 1.0f;
     const bool want_top_list = a.num_top > 0;
     bool have_hist = false, have_mass = false;           // which value histograms are current
     auto build_hist = [&](bool with_cnt, bool with_mass) {
@@ -959,19 +951,59 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         __syncthreads();
         have_hist = with_cnt; have_mass = with_mass;
     };
+    // The top-N list: the first min(num_top, members) entries, in order, of the set { C >= floorC } (the
+    // final kept set of `members` elements; in the full-vocabulary mode every finite score of the row).
+    auto write_top_list = [&](u64 members, u64 floorC, double lnS) {
+        const u64 want = members < (u64)a.num_top ? members : (u64)a.num_top;
+        u64 CN = floorC;
+        if (want < members) {
+            if (!have_hist) build_hist(true, false);
+            int bin; u64 cb, mb;
+            bool clobbered = false;
+            if (find_prefix_bin(s, h, false, false, want, bin, cb, mb))
+                CN = resolve_cut<DT>(s, h, c, zmax, bin, false, want, cb, floorC, clobbered);
+            if (clobbered) have_hist = have_mass = false;
+        }
+        u64 lo, hi;
+        const int n = gather_if<DT>(s, h, c, [&](u64 C, float) { return C >= CN && (C >> 32) < KEY_POS_INF; }, lo, hi);
+        const int m = n < ALBIREO_MAX_NUM_TOP ? n : ALBIREO_MAX_NUM_TOP;
+        if ((int)threadIdx.x < m) {
+            const u64 C = h.list[threadIdx.x];
+            int rank = 0;
+            for (int q = 0; q < m; ++q) rank += h.list[q] > C;
+            if (rank < a.num_top) {
+                const int64_t o = (int64_t)b * a.num_top + rank;
+                a.out_top_ids[o] = comp_idx(C);
+                a.out_top_logprobs[o] = (members == 1 && !full_lp) ? 0.0f : (float)(((double)unkey((uint32_t)(C >> 32)) - (double)zmax) - lnS);
+            }
+        }
+        __syncthreads();
+    };
+    // Greedy rows (and rows with a single finite score) need the arg max only -- unless the list over
+    // the whole vocabulary is wanted: then they go through the cuts below as top_k = 1.
+    if ((rp.greedy || n_fin <= 1) && !(full_lp && want_top_list)) {
+        out.token = top_id(); out.logprob = 0.0f; out.n_keep = 1; out.n_topk = 1;
+        if (full_lp) out.logprob = (float)-(log((double)full_vocab_mass<DT>(s, c, zmax)) - LN2_40);
+        if (a.dbg_topk_ids && a.dbg_cap >= 1 && threadIdx.x == 0) a.dbg_topk_ids[(int64_t)b * a.dbg_cap] = out.token;
+        if (want_top_list && threadIdx.x == 0) {
+            a.out_top_ids[(int64_t)b * a.num_top] = out.token;
+            a.out_top_logprobs[(int64_t)b * a.num_top] = out.logprob;
+        }
+        return;
+    }
     if (want_k || want_topp) build_hist(want_k, want_topp);
 
     // top-k stage
     u64 C1 = Cfin;
     u64 n_topk = n_fin;
     if (want_k) {
-        n_topk = (u64)rp.top_k;
+        n_topk = (u64)top_k;
         int bin; u64 cb, mb;
         const bool find_ok = find_prefix_bin(s, h, false, want_topp, n_topk, bin, cb, mb);
         bool clobbered = false;
         if (find_ok) C1 = resolve_cut<DT>(s, h, c, zmax, bin, false, n_topk, cb, Cfin, clobbered);
         if (clobbered) have_hist = have_mass = false;
-        if (a.flags & ALBIREO_FLAG_TOPK_KEEP_TIES) {
+        if ((a.flags & ALBIREO_FLAG_TOPK_KEEP_TIES) && !rp.greedy) {
             // every id of the k-th largest key stays; how many that makes takes a count over the row
             C1 &= 0xFFFFFFFF00000000ull;
             const uint32_t k1 = (uint32_t)(C1 >> 32);
@@ -982,7 +1014,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
         if (want_topp && !have_mass) build_hist(false, true);
     }
     out.n_topk = (int32_t)n_topk;
-    if (a.dbg_topk_ids && rp.top_k >= 1 && rp.top_k < V && n_topk <= (u64)a.dbg_cap) {
+    if (a.dbg_topk_ids && top_k >= 1 && top_k < V && n_topk <= (u64)a.dbg_cap) {
         if (threadIdx.x == 0) s.list_cnt = 0;
         __syncthreads();
         int32_t *dst = a.dbg_topk_ids + (int64_t)b * a.dbg_cap;
@@ -1106,32 +1138,7 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     out.logprob = (n_keep == 1 && !full_lp) ? 0.0f : (float)(((double)z_tok - (double)zmax) - lnS);
     out.n_keep = (int32_t)n_keep;
 
-    if (want_top_list) {
-        // first min(num_top, n_keep) entries of the kept set, in order
-        const u64 want = n_keep < (u64)a.num_top ? n_keep : (u64)a.num_top;
-        u64 CN = C2;
-        if (want < n_keep) {
-            if (!have_hist) build_hist(true, false);
-            int bin; u64 cb, mb;
-            bool clobbered = false;
-            if (find_prefix_bin(s, h, false, false, want, bin, cb, mb))
-                CN = resolve_cut<DT>(s, h, c, zmax, bin, false, want, cb, C2, clobbered);
-        }
-        u64 lo, hi;
-        const int n = gather_if<DT>(s, h, c, [&](u64 C, float) { return C >= CN; }, lo, hi);
-        const int m = n < ALBIREO_MAX_NUM_TOP ? n : ALBIREO_MAX_NUM_TOP;
-        if ((int)threadIdx.x < m) {
-            const u64 C = h.list[threadIdx.x];
-            int rank = 0;
-            for (int q = 0; q < m; ++q) rank += h.list[q] > C;
-            if (rank < a.num_top) {
-                const int64_t o = (int64_t)b * a.num_top + rank;
-                a.out_top_ids[o] = comp_idx(C);
-                a.out_top_logprobs[o] = (n_keep == 1 && !full_lp) ? 0.0f : (float)(((double)unkey((uint32_t)(C >> 32)) - (double)zmax) - lnS);
-            }
-        }
-        __syncthreads();
-    }
+    if (want_top_list) write_top_list(full_lp ? (u64)s.nfin_cap : n_keep, full_lp ? ((u64)KEY_MIN_FINITE << 32) : C2, lnS);
 }
 
 // ------------------------------------------------------------------ TMA bulk-copy ring
@@ -1538,7 +1545,10 @@ __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c
 }
 
 // which rows the candidate path takes (decided from the row's parameters alone)
-__device__ __forceinline__ bool candidate_eligible(const RowParams &rp, int V) {
+// (a top-N list over the whole vocabulary is the general path's business: the candidate list ends
+// where the cuts end)
+__device__ __forceinline__ bool candidate_eligible(const RowParams &rp, int V, bool full_list) {
+    if (full_list) return false;
     const int k = rp.greedy ? 1 : rp.top_k;
     const bool has_topk = rp.greedy || (k >= 1 && k < V);
     const bool has_minp = !rp.greedy && rp.min_p > 0.0f;
@@ -1900,7 +1910,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     c.has_hist = false; c.bitmap = nullptr; c.coarse = nullptr; c.counts = nullptr; c.n_distinct = 0; c.ncoarse = 0;
     if (!(c.r > 0.0f)) out.status |= ALBIREO_ROW_BAD_PARAM;
 
-    const bool try_candidates = ring_started && candidate_eligible(rp, V);
+    const bool try_candidates = ring_started && candidate_eligible(rp, V, (a.flags & ALBIREO_FLAG_LOGPROB_FULL_VOCAB) && a.num_top > 0);
     if (a.hist_ids && a.hist_off) {
         const int o0 = a.hist_off[b], o1 = a.hist_off[b + 1];
         if (o1 > o0) {

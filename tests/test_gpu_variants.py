@@ -349,6 +349,22 @@ def test_full_vocabulary_logprobs(binding, sampler, dtype, general):
     assert (plain.tokens == ref.tokens).all() and (ref.logprobs < plain.logprobs - 1e-9).sum() >= 20
 
 
+def test_full_vocabulary_top_list_reaches_past_the_cuts(binding, sampler):
+    """top_k below num_top, greedy rows, min-p only rows: the list is still the head of the whole row."""
+    w = W.random_small(802, B=40, V=6000, dtype=W.BF16)
+    w.top_k[:] = np.where(np.arange(40) % 3 == 0, 2, w.top_k)        # cuts far tighter than the list
+    w.logprob_full_vocab = True
+    w.num_top = 12
+    for general in (0, 1):
+        flags = binding.FLAG_LOGPROB_FULL_VOCAB | (binding.FLAG_FORCE_GENERAL if general else 0)
+        g, ref = check(binding, sampler, w, flags=flags)
+        assert (ref.top_ids >= 0).all() and (g["top_ids"] == ref.top_ids).all()
+    wk = W.random_small(802, B=40, V=6000, dtype=W.BF16)
+    wk.top_k[:] = np.where(np.arange(40) % 3 == 0, 2, wk.top_k)
+    wk.logprob_full_vocab = True; wk.topk_keep_ties = True; wk.num_top = 12
+    check(binding, sampler, wk, flags=binding.FLAG_LOGPROB_FULL_VOCAB | binding.FLAG_TOPK_KEEP_TIES)
+
+
 def test_full_vocabulary_logprobs_full_size_rows(binding, sampler):
     w = W.config4(B=48)
     w.logprob_full_vocab = True

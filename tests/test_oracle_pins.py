@@ -638,16 +638,19 @@ def test_full_vocabulary_logprobs_equal_library_log_softmax_whatever_the_cuts():
     x[3, ::7] = -np.inf                                     # masked entries carry no mass
     T = np.float32(0.8)
     ref = scipy.special.log_softmax((x * (np.float32(1.0) / T)).astype(np.float64), axis=1)
-    base = O.sample(one_row(x, T=float(T), top_k=20, top_p=0.9, min_p=0.02, seed=4, num_top=6))
-    w = one_row(x, T=float(T), top_k=20, top_p=0.9, min_p=0.02, seed=4, num_top=6)
+    base = O.sample(one_row(x, T=float(T), top_k=3, top_p=0.9, min_p=0.02, seed=4, num_top=6))
+    w = one_row(x, T=float(T), top_k=3, top_p=0.9, min_p=0.02, seed=4, num_top=6)
     w.logprob_full_vocab = True
     o = O.sample(w)
     assert (o.tokens == base.tokens).all() and (o.rows["n_keep"] == base.rows["n_keep"]).all()   # the draw is untouched
     for b in range(B):
         assert abs(o.logprobs[b] - ref[b, o.tokens[b]]) < 1e-12
+        # the list is the head of the whole row's order, whatever the cuts kept
+        zb = (x[b] * (np.float32(1.0) / T)).astype(np.float64)
+        want = np.lexsort((np.arange(V), -zb))[:6]
+        assert o.top_ids[b].tolist() == want.tolist()
         for j in range(6):
-            if o.top_ids[b, j] >= 0:
-                assert abs(o.top_logprobs[b, j] - ref[b, o.top_ids[b, j]]) < 1e-12
+            assert abs(o.top_logprobs[b, j] - ref[b, o.top_ids[b, j]]) < 1e-12
         assert o.logprobs[b] <= base.logprobs[b] + 1e-15      # the kept set's normaliser is the smaller one
     # greedy rows: the arg max under the softmax of the unscaled scores
     g = one_row(x, T=0.0)
