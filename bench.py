@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of albireo_sample_kernel on the
 # metric workload, from the ncu capture summarised in profiles/albireo_sample_kernel_configM.md
 # (mean of the two captured launches).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"configM": 79494656}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"configM": 79677824}
 
 
 def measured_peak():
