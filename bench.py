@@ -235,6 +235,9 @@ def main():
     ap.add_argument("--sequence-parallel", default=None, choices=["a2a", "gather"],
                     help="secondary mode: logits start as per-rank vocabulary shards; time all-to-all + sample + "
                          "gather (a2a) or the gather-to-one-rank arrangement it replaces (gather)")
+    ap.add_argument("--pdl", action="store_true",
+                    help="launch every call with programmatic stream serialisation (ALBIREO_FLAG_PROGRAMMATIC_LAUNCH): "
+                         "a call's launch overlaps the tail of the call before it; off by default")
     ap.add_argument("--read-ceiling", action="store_true",
                     help="only run the read-ceiling tool (a kernel that just reads the same bytes) and print its table")
     args = ap.parse_args()
@@ -292,6 +295,8 @@ def main():
     flags = binding.FLAG_FORCE_GENERAL if args.general_path else 0
     if args.variant == "fullvocab":
         flags |= binding.FLAG_LOGPROB_FULL_VOCAB
+    if args.pdl:
+        flags |= binding.FLAG_PROGRAMMATIC_LAUNCH
     stream = torch.cuda.Stream(device=dev)
     if args.variant == "feedback":
         t["backfill_ids"] = torch.zeros(w.backfill_len, dtype=torch.int32, device=dev)
@@ -402,6 +407,7 @@ def main():
                 "launch": "one CUDA graph of K launches" if graph is not None else "K launches from the host",
                 "path": "general path forced" if args.general_path else "automatic",
                 "variant": args.variant,
+                "programmatic_launch": bool(args.pdl),
             },
             "tokens_per_s": value,
             "roofline": {

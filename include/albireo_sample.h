@@ -77,6 +77,12 @@ enum {
                                          top-N list (num_top > 0) then holds the first entries of the
                                          whole row's order, not of the kept set; rows with such a
                                          list take the general path                               */
+#define ALBIREO_FLAG_PROGRAMMATIC_LAUNCH 8u /* launch with programmatic stream serialisation: the
+                                         kernel's CTAs may be scheduled while the kernel ahead of it
+                                         in the stream is still running (its launch latency and CTA
+                                         scheduling then overlap that kernel's tail); each CTA waits
+                                         for that kernel to complete before it reads or writes
+                                         anything, so the results are unchanged                      */
 
 /*
  * Optional arguments of albireo_sample (pass NULL for all defaults).  Zero-initialise,

@@ -31,6 +31,7 @@ ROW_GENERAL_PATH, ROW_BAD_PARAM, ROW_HISTORY_OVERFLOW, ROW_TIMEOUT = 1, 2, 4, 8
 FLAG_FORCE_GENERAL = 1
 FLAG_TOPK_KEEP_TIES = 2
 FLAG_LOGPROB_FULL_VOCAB = 4
+FLAG_PROGRAMMATIC_LAUNCH = 8
 MAX_VOCAB = 524288
 MAX_NUM_TOP = 128
 FIXED_MAX_HISTORY = 1 << 20

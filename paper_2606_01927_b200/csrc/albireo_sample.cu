@@ -1845,6 +1845,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     }
     out.n_topk = n_topk;
     const u64 full_fx = (a.flags & ALBIREO_FLAG_LOGPROB_FULL_VOCAB) ? full_vocab_mass<DT>(s, c, unkey(kmax)) : 0ull;
+    // the stream is over: a dependent kernel launched the same way may be scheduled from here on
+    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     final_stage(s, cs, n, L6, unkey(kmax), has_minp, rp, a, b, out, full_fx);
     return true;
 }
@@ -1875,6 +1877,9 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     // The ring is started before anything else is read, the row's own parameters included: their
     // loads and the first tiles then travel together.  A row that turns out to need the general
     // path waits for these copies before it reuses the shared memory.
+    // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
+    // stream (the producer of the logits) was still running: wait for it before anything is read or written.
+    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.wait;" ::: "memory");
     const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
     if (ring_started) candidate_begin<DT>(s, rg, c);
 
@@ -2044,6 +2049,20 @@ int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, cons
 }
 
 void launch_sample_kernel(int dtype, int B, size_t smem, cudaStream_t st, const SampleArgs &a) {
+    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) {
+        // programmatic dependent launch: the kernel may be scheduled before the kernel ahead of it in the
+        // stream has finished; it waits for that kernel itself (griddepcontrol.wait) before it touches memory
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)B); cfg.blockDim = dim3(NT); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        if (dtype == ALBIREO_F32) cudaLaunchKernelEx(&cfg, albireo_sample_kernel<ALBIREO_F32>, a);
+        else if (dtype == ALBIREO_BF16) cudaLaunchKernelEx(&cfg, albireo_sample_kernel<ALBIREO_BF16>, a);
+        else cudaLaunchKernelEx(&cfg, albireo_sample_kernel<ALBIREO_F16>, a);
+        return;
+    }
     if (dtype == ALBIREO_F32) albireo_sample_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(a);
     else if (dtype == ALBIREO_BF16) albireo_sample_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(a);
     else albireo_sample_kernel<ALBIREO_F16><<<B, NT, smem, st>>>(a);

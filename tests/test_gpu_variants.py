@@ -369,3 +369,34 @@ def test_full_vocabulary_logprobs_full_size_rows(binding, sampler):
     w = W.config4(B=48)
     w.logprob_full_vocab = True
     check(binding, sampler, w, flags=binding.FLAG_LOGPROB_FULL_VOCAB)
+
+
+# ------------------------------------------------------------------ programmatic dependent launch
+
+def test_programmatic_launch_gives_the_same_results(binding, sampler):
+    """Back-to-back calls launched with programmatic stream serialisation, the second reading what the
+    first wrote nowhere: each equals the plain launch bit for bit, also inside a captured graph."""
+    w = W.config3(B=32)
+    t = binding.workload_tensors(w, sampler.device)
+    lg = t.pop("logits")
+    plain = sampler.albireo_sample(lg, **t, num_top=4)
+    torch.cuda.synchronize()
+    outs = [sampler.albireo_sample(lg, **t, num_top=4, flags=binding.FLAG_PROGRAMMATIC_LAUNCH) for _ in range(4)]
+    torch.cuda.synchronize()
+    for o in outs:
+        assert torch.equal(o.tokens, plain.tokens) and torch.equal(o.logprobs, plain.logprobs)
+        assert torch.equal(o.top_ids, plain.top_ids)
+    st = torch.cuda.Stream(device=sampler.device)
+    tok = torch.empty(32, dtype=torch.int32, device=sampler.device)
+    lp = torch.empty(32, dtype=torch.float32, device=sampler.device)
+    with torch.cuda.stream(st):
+        sampler.albireo_sample(lg, **t, out_tokens=tok, out_logprobs=lp, stream=st, flags=binding.FLAG_PROGRAMMATIC_LAUNCH)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        for _ in range(3):
+            sampler.albireo_sample(lg, **t, out_tokens=tok, out_logprobs=lp, stream=st, flags=binding.FLAG_PROGRAMMATIC_LAUNCH)
+    tok.fill_(-9)
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(tok, plain.tokens) and torch.equal(lp, plain.logprobs)
