@@ -89,7 +89,8 @@ def test_binding_struct_and_constants_match_the_header(tmp_path):
             '  printf("sizeof %zu\\n", sizeof(albireo_sample_ext_t));']
     prog += [f'  printf("{f} %zu\\n", offsetof(albireo_sample_ext_t, {f}));' for f in fields]
     for name in ("ALBIREO_F32", "ALBIREO_BF16", "ALBIREO_F16", "ALBIREO_MAX_VOCAB", "ALBIREO_MAX_NUM_TOP",
-                 "ALBIREO_FLAG_FORCE_GENERAL", "ALBIREO_FLAG_TOPK_KEEP_TIES", "ALBIREO_FIXED_MAX_HISTORY", "ALBIREO_OK"):
+                 "ALBIREO_FLAG_FORCE_GENERAL", "ALBIREO_FLAG_TOPK_KEEP_TIES", "ALBIREO_FLAG_LOGPROB_FULL_VOCAB",
+                 "ALBIREO_FLAG_PROGRAMMATIC_LAUNCH", "ALBIREO_FIXED_MAX_HISTORY", "ALBIREO_OK"):
         prog.append(f'  printf("{name} %lld\\n", (long long){name});')
     prog += ['  return 0;', '}']
     src = tmp_path / "layout.c"
@@ -104,4 +105,6 @@ def test_binding_struct_and_constants_match_the_header(tmp_path):
     assert int(out["ALBIREO_MAX_VOCAB"]) == binding.MAX_VOCAB and int(out["ALBIREO_MAX_NUM_TOP"]) == binding.MAX_NUM_TOP
     assert int(out["ALBIREO_FLAG_FORCE_GENERAL"]) == binding.FLAG_FORCE_GENERAL
     assert int(out["ALBIREO_FLAG_TOPK_KEEP_TIES"]) == binding.FLAG_TOPK_KEEP_TIES
+    assert int(out["ALBIREO_FLAG_LOGPROB_FULL_VOCAB"]) == binding.FLAG_LOGPROB_FULL_VOCAB
+    assert int(out["ALBIREO_FLAG_PROGRAMMATIC_LAUNCH"]) == binding.FLAG_PROGRAMMATIC_LAUNCH
     assert int(out["ALBIREO_FIXED_MAX_HISTORY"]) == binding.FIXED_MAX_HISTORY and int(out["ALBIREO_OK"]) == binding.OK
