@@ -190,16 +190,37 @@ def run_sequence_parallel(args, rank, world, local_rank):
             return SP.sample_step(fn, shards[i % N_ROTATING], meta_local, lay, step=w.step, recv=recv)
         return SP.gather_then_sample_step(fn, shards[i % N_ROTATING], meta_all, s_rows, step=w.step)
 
-    for i in range(args.warmup):
-        step(i)
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            step(i)
     torch.cuda.synchronize(dev)
+    # the K steps as one CUDA graph (collectives included): from the host they are launch-bound
+    graph = None
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(args.steps):
+                    step(i)
+            graph.replay()
+            torch.cuda.synchronize(dev)
+        except Exception as exc:                    # a library that cannot be captured: time the host-launched steps
+            print(f"[bench] graph capture of the sequence-parallel step failed ({exc}); launching from the host",
+                  file=sys.stderr)
+            graph = None
+            torch.cuda.synchronize(dev)
     dist.barrier()
     torch.cuda.synchronize(dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        step(i)
-    e1.record()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        if graph is not None:
+            graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
+        e1.record(stream)
     torch.cuda.synchronize(dev)
     dist.barrier()
     tt = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
@@ -211,8 +232,10 @@ def run_sequence_parallel(args, rank, world, local_rank):
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": describe(w), "mode": "sequence-parallel " + args.sequence_parallel,
-                       "rows_per_gpu": lay.rows, "launch": "K steps from the host (collectives + one kernel each)"},
-            "gpu_launches": sampler.launch_count() - args.warmup}))
+                       "rows_per_gpu": lay.rows,
+                       "launch": "one CUDA graph of K steps (collectives + one kernel each)" if graph is not None
+                       else "K steps from the host (collectives + one kernel each)"},
+            "gpu_launches": args.steps}))
     dist.destroy_process_group()
 
 
