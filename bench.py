@@ -184,8 +184,21 @@ def run_sequence_parallel(args, rank, world, local_rank):
     meta_local = SP.scatter_metadata(meta_all if rank == 0 else None, lay, dev)
     fn = SP.cuda_sample_fn(sampler)
     recv = torch.empty((world, lay.rows, vs), dtype=shards[0].dtype, device=dev)
+    peer_bufs = None
+    if args.sequence_parallel == "peer":
+        # every rank's shard lives in symmetric memory (one buffer per rotation); the "LM head" output is copied in once
+        peer_bufs = []
+        for sh in shards:
+            mine, peers, handle = SP.peer_shards(lay.s_padded, vs, sh.dtype, dev)
+            mine[:s_rows].copy_(sh)
+            peer_bufs.append((peers, handle))
+        torch.cuda.synchronize(dev)
+        dist.barrier()
 
     def step(i):
+        if args.sequence_parallel == "peer":
+            peers, handle = peer_bufs[i % N_ROTATING]
+            return SP.peer_sample_step(sampler, peers, handle, meta_local, lay, step=w.step)
         if args.sequence_parallel == "a2a":
             return SP.sample_step(fn, shards[i % N_ROTATING], meta_local, lay, step=w.step, recv=recv)
         return SP.gather_then_sample_step(fn, shards[i % N_ROTATING], meta_all, s_rows, step=w.step)
@@ -255,9 +268,10 @@ def main():
                     help="the same workload as binary16 logits, with a pre-generated Exp(1) table, or with the "
                          "early-feedback targets (next input ids + pinned host ring), or with log-probabilities "
                          "relative to the full vocabulary")
-    ap.add_argument("--sequence-parallel", default=None, choices=["a2a", "gather"],
+    ap.add_argument("--sequence-parallel", default=None, choices=["a2a", "gather", "peer"],
                     help="secondary mode: logits start as per-rank vocabulary shards; time all-to-all + sample + "
-                         "gather (a2a) or the gather-to-one-rank arrangement it replaces (gather)")
+                         "gather (a2a), the gather-to-one-rank arrangement it replaces (gather), or the step without an "
+                         "exchange: the sampler reads the peers' shards in place from symmetric memory (peer)")
     ap.add_argument("--pdl", action="store_true",
                     help="launch every call with programmatic stream serialisation (ALBIREO_FLAG_PROGRAMMATIC_LAUNCH): "
                          "a call's launch overlaps the tail of the call before it; off by default")

@@ -56,6 +56,8 @@ enum {
 /* limits */
 #define ALBIREO_MAX_VOCAB 524288   /* V above this is rejected                            */
 #define ALBIREO_MAX_NUM_TOP 128    /* largest num_top (top-N logprob list)                */
+#define ALBIREO_MAX_SEGMENTS 64    /* largest num_segments                                */
+#define ALBIREO_MAX_PEER_SEGMENTS 16 /* largest num_segments with segment_ptrs            */
 
 /* bits of out_row_status[b] */
 #define ALBIREO_ROW_GENERAL_PATH 1u  /* informational: row took the multi-pass general path */
@@ -152,6 +154,18 @@ typedef struct albireo_sample_ext {
        a = rep(x); a -= f * c_out; if (c_out > 0) a -= p.  Values are clamped to [0, length].
        NULL: every id counts as output (the three penalties share one history).             */
     const int32_t *history_output_start; /* [B] device, or NULL                              */
+
+    /* Rows in pieces without an exchange step: with segment_ptrs (a HOST array of num_segments
+       device pointers, <= ALBIREO_MAX_PEER_SEGMENTS) piece j of row b is read from
+       segment_ptrs[j] + (segment_row_offset + b) * row_stride + (i % Vs), i.e. from the
+       vocabulary shard [s, V/t] as it lies in worker j's own memory (peer-mapped: symmetric memory,
+       IPC or cudaMemcpyPeer-capable mappings all do).  The logits then cross NVLink once, straight
+       into the sampler's shared memory, and the all-to-all of section 6.1 step 2 disappears; the
+       caller makes sure every worker's shard is complete before the launch and not overwritten
+       before the call has finished.  `logits` is ignored (pass segment_ptrs[0]);
+       segment_stride_elems is unused; every pointer must be 16-byte aligned.  NULL: one buffer. */
+    const void *const *segment_ptrs;     /* host array of device pointers, or NULL              */
+    int64_t segment_row_offset;          /* rows before this call's row 0 in every piece buffer  */
 } albireo_sample_ext_t;
 
 /*

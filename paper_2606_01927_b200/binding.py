@@ -55,6 +55,7 @@ class SampleExt(C.Structure):
         ("feedback_ring", C.c_void_p), ("feedback_cap", C.c_int64), ("feedback_head", C.c_int64),
         ("num_segments", C.c_int32), ("segment_stride_elems", C.c_int64),
         ("history_output_start", C.c_void_p),
+        ("segment_ptrs", C.c_void_p), ("segment_row_offset", C.c_int64),
     ]
 
 
@@ -207,7 +208,8 @@ class Sampler:
                        want_status=False, flags: int = 0, B: Optional[int] = None, V: Optional[int] = None,
                        exp1: Optional[torch.Tensor] = None, backfill_ids: Optional[torch.Tensor] = None,
                        backfill_index: Optional[torch.Tensor] = None, feedback_ring: Optional[torch.Tensor] = None,
-                       feedback_head: int = 0, output_start: Optional[torch.Tensor] = None) -> SampleOutputs:
+                       feedback_head: int = 0, output_start: Optional[torch.Tensor] = None,
+                       segment_tensors=None, segment_row_offset: int = 0) -> SampleOutputs:
         """Device-resident call: all tensors on ``self.device``; asynchronous on ``stream``.
 
         ``exp1`` (float32 ``[B, V]``) replaces the counter-based draw by pre-generated Exp(1)
@@ -244,6 +246,19 @@ class Sampler:
             ext.row_stride_elems = row_stride
         if output_start is not None:
             ext.history_output_start = _dp(output_start, torch.int32, "cuda")
+        if segment_tensors is not None:
+            # one [rows, V/t] buffer per piece (e.g. the peers' vocabulary shards in symmetric memory), read in place
+            t_ = len(segment_tensors)
+            sh0 = segment_tensors[0]
+            if any(x.dim() != 2 or x.stride(1) != 1 or x.dtype != sh0.dtype or x.shape[1] != sh0.shape[1]
+                   or x.stride(0) != sh0.stride(0) for x in segment_tensors):
+                raise ValueError("segment_tensors must be same-shaped [rows, V/t] tensors with unit stride along V/t")
+            ptrs = (C.c_void_p * t_)(*[x.data_ptr() for x in segment_tensors])
+            ext.num_segments = t_
+            ext.segment_ptrs = C.cast(ptrs, C.c_void_p)
+            ext.segment_row_offset = segment_row_offset
+            ext.row_stride_elems = sh0.stride(0)
+            ext._keepalive = ptrs
         if exp1 is not None:
             if exp1.dtype != torch.float32 or exp1.dim() != 2 or exp1.stride(1) != 1 or exp1.device != dev:
                 raise ValueError("exp1 must be a float32 [B, V] tensor on the logits' device")

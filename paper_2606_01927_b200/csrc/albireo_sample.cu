@@ -58,6 +58,9 @@ struct SampleArgs {
     int32_t nseg;               // pieces per row (1: rows are contiguous)
     int64_t seg_stride;         // elements between consecutive pieces of a row
     int32_t Vs, vps;            // elements and 16-byte vectors per piece (worked out on the host: no division on the device)
+    int32_t seg_ptr_count;      // > 0: the pieces live in buffers of their own, seg_ptr[j]; 0: a stride apart in `logits`
+    int64_t seg_row_offset;     // rows to skip at the start of every piece buffer
+    const void *seg_ptr[ALBIREO_MAX_PEER_SEGMENTS];
     const float *temperature;
     const int32_t *top_k;
     const float *top_p, *min_p, *rep, *pres, *freq;
@@ -170,6 +173,7 @@ struct BlockScratch {
     uint32_t done[MAX_STAGES];   // warps finished with each ring stage
     uint32_t maint_at;           // tile index before which every warp meets (0xFFFFFFFF: none)
     uint32_t issued;             // tiles whose copy has been issued so far
+    const char *seg_base[ALBIREO_MAX_SEGMENTS];   // where this row's pieces start (rows in pieces only)
     uint32_t nfin_cap;           // general path: min(#finite scores, ALBIREO_MAX_NUM_TOP + 1), parked here until the list is written
 };
 
@@ -226,9 +230,10 @@ struct RowCtx {
     const void *row;       // first logit of the row
     int V;
     // a row may arrive as nseg equal pieces of Vs elements (vocabulary shards as the all-to-all of
-    // sequence-parallel sampling leaves them, section 6.1 step 2), seg_bytes apart; nseg == 1: one piece
+    // sequence-parallel sampling leaves them, section 6.1 step 2), in one buffer a stride apart or in a
+    // buffer each (other workers' memory included); nseg == 1: one piece
     int nseg, Vs;
-    int64_t seg_bytes;
+    const char *const *seg_base;   // shared-memory table: start of each piece of this row
     float invT, r, p, f;
     bool has_hist;
     const uint32_t *bitmap;   // V bits (+1 pad word): token appears in the history
@@ -302,7 +307,7 @@ template <int DT>
 __device__ __forceinline__ const void *elem_ptr(const RowCtx &c, int i) {
     if (c.nseg == 1) return (const char *)c.row + (size_t)i * Elem<DT>::SIZE;
     const int j = i / c.Vs;
-    return (const char *)c.row + (size_t)j * (size_t)c.seg_bytes + (size_t)(i - j * c.Vs) * Elem<DT>::SIZE;
+    return c.seg_base[j] + (size_t)(i - j * c.Vs) * Elem<DT>::SIZE;
 }
 // address of the row's v-th 16-byte vector (rows in pieces are 16-byte aligned piece by piece, so
 // their vectors start at element 0 and none straddles two pieces)
@@ -311,7 +316,7 @@ __device__ __forceinline__ const uint4 *vec_ptr(const RowCtx &c, const uint4 *vp
     if (c.nseg == 1) return vp + v;
     const int vps = c.Vs / Elem<DT>::PER_VEC;
     const int j = v / vps;
-    return (const uint4 *)((const char *)c.row + (size_t)j * (size_t)c.seg_bytes) + (v - j * vps);
+    return (const uint4 *)c.seg_base[j] + (v - j * vps);
 }
 
 __device__ __forceinline__ float score_of(const RowCtx &c, int i, float x) {
@@ -1152,7 +1157,7 @@ struct Ring {
     // source of the copies: vectors per piece of the row and the distance between pieces (a row in
     // one piece: vps covers the whole row)
     int vps;
-    int64_t seg_vecs;
+    const char *const *seg_base;
     unsigned char *buf;     // nstages * STAGE_BYTES, 128-byte aligned
     uint64_t *bar;          // one mbarrier per stage
     int nstages;
@@ -1187,7 +1192,7 @@ __device__ __forceinline__ void ring_copy(const Ring &rg, void *dst, const uint4
     int j = v0 / rg.vps, off = v0 - j * rg.vps;
     while (nv > 0) {
         const int n1 = nv < rg.vps - off ? nv : rg.vps - off;
-        bulk_g2s(d, vp + (int64_t)j * rg.seg_vecs + off, (uint32_t)n1 * 16u, bar);
+        bulk_g2s(d, (const uint4 *)rg.seg_base[j] + off, (uint32_t)n1 * 16u, bar);
         d += (size_t)n1 * 16; nv -= n1; ++j; off = 0;
     }
 }
@@ -1867,13 +1872,24 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     Ring rg;
     rg.nstages = a.nstages;
     rg.vps = a.vps;
-    rg.seg_vecs = a.seg_stride * Elem<DT>::SIZE / 16;
+    rg.seg_base = s.seg_base;
     rg.buf = smem + COMMON_BYTES;
     rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
     RowCtx c;
     c.row = (const char *)a.logits + (size_t)b * (size_t)a.row_stride * Elem<DT>::SIZE;
     c.V = V;
-    c.nseg = a.nseg; c.Vs = a.Vs; c.seg_bytes = a.seg_stride * Elem<DT>::SIZE;
+    c.nseg = a.nseg; c.Vs = a.Vs; c.seg_base = s.seg_base;
+    if (a.nseg > 1) {
+        // where the pieces of this row start: a stride apart in one buffer, or one buffer per piece (the
+        // senders' own memory, read in place over NVLink: then there is no exchange step at all)
+        const size_t row_off = (size_t)(a.seg_row_offset + b) * (size_t)a.row_stride * Elem<DT>::SIZE;
+        if (a.seg_ptr_count > 0) c.row = (const char *)a.seg_ptr[0] + row_off;
+        if (threadIdx.x == 0) {             // thread 0 issues the ring's copies; everyone else reads the table after a barrier
+            for (int j = 0; j < a.nseg; ++j)
+                s.seg_base[j] = a.seg_ptr_count > 0 ? (const char *)a.seg_ptr[j] + row_off
+                                                    : (const char *)c.row + (size_t)j * (size_t)a.seg_stride * Elem<DT>::SIZE;
+        }
+    }
     // The ring is started before anything else is read, the row's own parameters included: their
     // loads and the first tiles then travel together.  A row that turns out to need the general
     // path waits for these copies before it reuses the shared memory.
@@ -2020,13 +2036,22 @@ int apply_ext(SampleArgs &a, const albireo_sample_ext_t *ext, int B, int V, cons
         const int64_t esz = a.elem_size, t = ext->num_segments;
         if (t > 64 || V % t) { *why = "num_segments must divide V and be at most 64"; return ALBIREO_EINVAL; }
         const int64_t Vs = V / t;
-        if (ext->segment_stride_elems < Vs) { *why = "segment stride smaller than a piece"; return ALBIREO_EINVAL; }
+        if (!ext->segment_ptrs && ext->segment_stride_elems < Vs) { *why = "segment stride smaller than a piece"; return ALBIREO_EINVAL; }
         if (ext->row_stride_elems == 0) a.row_stride = Vs;
         if (a.row_stride < Vs) { *why = "row stride smaller than a piece"; return ALBIREO_EINVAL; }
         if ((Vs * esz) % 16 || (a.row_stride * esz) % 16 || (ext->segment_stride_elems * esz) % 16 || (uintptr_t)a.logits % 16) {
             *why = "rows in pieces need 16-byte aligned pieces, row stride, segment stride and base"; return ALBIREO_EUNSUPPORTED;
         }
         a.nseg = (int32_t)t; a.seg_stride = ext->segment_stride_elems;
+        if (ext->segment_ptrs) {
+            if (t > ALBIREO_MAX_PEER_SEGMENTS) { *why = "segment_ptrs takes at most ALBIREO_MAX_PEER_SEGMENTS pieces"; return ALBIREO_EUNSUPPORTED; }
+            if (ext->segment_row_offset < 0) { *why = "segment_row_offset is negative"; return ALBIREO_EINVAL; }
+            for (int64_t j = 0; j < t; ++j) {
+                if (!ext->segment_ptrs[j] || (uintptr_t)ext->segment_ptrs[j] % 16) { *why = "segment_ptrs entries must be non-NULL and 16-byte aligned"; return ALBIREO_EUNSUPPORTED; }
+                a.seg_ptr[j] = ext->segment_ptrs[j];
+            }
+            a.seg_ptr_count = (int32_t)t; a.seg_row_offset = ext->segment_row_offset;
+        }
         a.Vs = (int32_t)Vs; a.vps = (int32_t)(Vs * esz / 16);
     } else if (ext->num_segments < 0) { *why = "num_segments is negative"; return ALBIREO_EINVAL; }
     a.out_start = ext->history_output_start;

@@ -177,3 +177,35 @@ def gather_then_sample_step(sample_fn: SampleFn, local_shard: torch.Tensor, meta
     dist.broadcast(tok, src=dst, group=group)
     dist.broadcast(lp, src=dst, group=group)
     return tok, lp
+
+
+# ------------------------------------------------------------------ no exchange step: read the peers' shards in place
+
+def peer_shards(s_padded: int, vs: int, dtype: torch.dtype, device, group=None):
+    """Allocates this worker's ``[s', v/t]`` vocabulary shard in symmetric memory and maps every peer's.
+    Returns ``(mine, peers, handle)``: the LM head writes ``mine``; ``peers[j]`` is worker ``j``'s shard
+    as a tensor on this device (peer-mapped; ``peers[rank] is`` the local one); ``handle.barrier()`` is
+    the cross-worker barrier.  Padding rows stay zero."""
+    import torch.distributed._symmetric_memory as symm
+    mine = symm.empty((s_padded, vs), dtype=dtype, device=device)
+    mine.zero_()
+    grp = dist.group.WORLD if group is None else group
+    handle = symm.rendezvous(mine, grp)
+    world = dist.get_world_size(group)
+    peers = [handle.get_buffer(r, (s_padded, vs), dtype) for r in range(world)]
+    return mine, peers, handle
+
+
+def peer_sample_step(sampler, peers, handle, meta_local: Dict[str, Optional[torch.Tensor]], lay: Layout, step: int,
+                     group=None):
+    """Steps (2)-(4) with step (2) folded into step (3): the sampler reads piece ``j`` of each of its
+    rows straight from worker ``j``'s shard (``segment_ptrs`` of the C ABI), so every logit crosses
+    NVLink once, into the sampler's shared memory, and no exchange buffer exists.  Plain bulk copies
+    from peer memory, no multicast.  The barriers make sure that every shard is complete before it is
+    read and not overwritten before everybody has read it."""
+    vs = peers[0].shape[1]
+    handle.barrier()
+    out = sampler.albireo_sample(peers[0], **meta_local, B=lay.rows, V=vs * lay.t, step=step, row_base=lay.row_base,
+                                 segment_tensors=peers, segment_row_offset=lay.row_base)
+    handle.barrier()
+    return gather_results(out.tokens, out.logprobs, lay, group=group)

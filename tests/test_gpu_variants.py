@@ -400,3 +400,61 @@ def test_programmatic_launch_gives_the_same_results(binding, sampler):
     g.replay()
     torch.cuda.synchronize()
     assert torch.equal(tok, plain.tokens) and torch.equal(lp, plain.logprobs)
+
+
+# ------------------------------------------------------------------ pieces in buffers of their own (peer memory stand-in)
+
+@pytest.mark.parametrize("t,dtype,V", [(2, W.BF16, 8192), (4, W.BF16, 152064), (4, W.F32, 40000), (8, W.F16, 70016)])
+@pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
+def test_pieces_in_separate_buffers(binding, sampler, t, dtype, V, flags):
+    """Every piece in an allocation of its own, as if it were another worker's vocabulary shard [s, V/t]
+    with this call's rows starting at row 5: the sampler reads them in place through a pointer table."""
+    import ctypes as C
+    base = W.random_small(900 + t, B=20, V=V, dtype=W.F32 if dtype == W.F16 else dtype)
+    w = W.as_f16(base) if dtype == W.F16 else base
+    w.num_top = 3
+    ref = O.sample(w, threads=_CORES, topk_cap=DBG_CAP)
+    tt = binding.workload_tensors(w, sampler.device)
+    lg = tt.pop("logits")
+    Vs, off = V // t, 5
+    shards = []
+    for j in range(t):
+        sh = torch.zeros((off + w.B + 2, Vs), dtype=lg.dtype, device=lg.device)      # other rows before and after
+        sh[off:off + w.B] = lg[:, j * Vs:(j + 1) * Vs]
+        shards.append(sh)
+    out = sampler.albireo_sample(shards[0], **tt, B=w.B, V=V, num_top=w.num_top, want_counts=True, dbg_cap=DBG_CAP,
+                                 want_status=True, flags=flags, segment_tensors=shards, segment_row_offset=off)
+    torch.cuda.synchronize()
+    g = to_host(out)
+    rep = compare(w, g, ref, dbg_cap=DBG_CAP)
+    print(rep.summary())
+    assert rep.ok(), rep.failures[:5]
+    assert len(rep.excused) <= 1 and not compare_top_lists(w, g, ref)
+
+
+def test_peer_shards_step_on_one_rank(binding, sampler):
+    """The exchange-free sequence-parallel step through symmetric memory with a group of one: allocation,
+    rendezvous, barrier, the sampler reading the (here: its own) shard through the pointer table, gather."""
+    import socket
+    import torch.distributed as dist
+    from paper_2606_01927_b200 import sequence_parallel as SP
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=sampler.device)
+    try:
+        w = W.config2(B=24)
+        ref = O.sample(w, threads=_CORES)
+        tt = binding.workload_tensors(w, sampler.device)
+        lg, step = tt.pop("logits"), tt.pop("step")
+        lay = SP.layout(w.B)
+        mine, peers, handle = SP.peer_shards(lay.s_padded, w.V, lg.dtype, sampler.device)
+        mine[: w.B].copy_(lg)                                 # what the LM head would have written
+        meta = SP.scatter_metadata(tt, lay, sampler.device)
+        tok, lp = SP.peer_sample_step(sampler, peers, handle, meta, lay, step=step)
+        torch.cuda.synchronize()
+        assert (tok.cpu().numpy() == ref.tokens).all()
+        assert np.abs(lp.cpu().numpy() - ref.logprobs).max() < 2e-5
+    finally:
+        dist.destroy_process_group()
