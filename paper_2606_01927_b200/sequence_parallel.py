@@ -201,7 +201,7 @@ def peer_sample_step(sampler, peers, handle, meta_local: Dict[str, Optional[torc
     """Steps (2)-(4) with step (2) folded into step (3): the sampler reads piece ``j`` of each of its
     rows straight from worker ``j``'s shard (``segment_ptrs`` of the C ABI), so every logit crosses
     NVLink once, into the sampler's shared memory, and no exchange buffer exists.  Plain bulk copies
-    from peer memory, no multicast.  The barriers make sure that every shard is complete before it is
+    from peer memory, each CTA fetching its own tiles.  The barriers make sure that every shard is complete before it is
     read and not overwritten before everybody has read it."""
     vs = peers[0].shape[1]
     handle.barrier()
