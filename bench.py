@@ -255,7 +255,7 @@ def run_sequence_parallel(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="albireo", choices=["albireo", "reference"])
     ap.add_argument("--workload", default="configM")
