@@ -101,7 +101,7 @@ def compare(w, gpu, oracle_out, dbg_cap: int = 0, name: str = "") -> ParityRepor
 
 def compare_top_lists(w, gpu, oracle_out) -> list:
     """Top-N lists: same ids in the same order and logprobs within tolerance, for rows whose
-    final kept-set size agrees (otherwise the row is a cut-boundary case judged on token+logprob)."""
+    final kept-set size agrees (otherwise the row is a cut-boundary case checked on token+logprob)."""
     bad = []
     if not w.num_top:
         return bad

@@ -270,7 +270,7 @@ def test_sequence_parallel_step_on_one_rank(binding, sampler):
         meta = SP.scatter_metadata(tt, lay, sampler.device)
         tok, lp = SP.sample_step(SP.cuda_sample_fn(sampler), shard, meta, lay, step=step)
         torch.cuda.synchronize()
-        assert (tok.cpu().numpy() == ref.tokens).mean() >= 0.97          # cut-boundary rows are judged in the parity tests
+        assert (tok.cpu().numpy() == ref.tokens).mean() >= 0.97          # cut-boundary rows are dealt with in the parity tests
         assert np.abs(lp.cpu().numpy()[tok.cpu().numpy() == ref.tokens] - ref.logprobs[tok.cpu().numpy() == ref.tokens]).max() < 1e-4
     finally:
         dist.destroy_process_group()
