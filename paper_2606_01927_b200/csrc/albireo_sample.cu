@@ -52,35 +52,33 @@ constexpr float FX_SCALE = 1099511627776.0f;       // 2^40: fixed-point scale of
 constexpr double LN2_40 = 27.725887222397812;      // 40 ln 2
 
 struct SampleArgs {
+    // (ordered by first use: a launch's arguments sit in constant memory no SM has seen before, and
+    // every 64-byte line of them costs a miss at first touch)
     const void *logits;
     int32_t B, V;
     int64_t row_stride;
     int32_t nseg;               // pieces per row (1: rows are contiguous)
-    int64_t seg_stride;         // elements between consecutive pieces of a row
-    int32_t Vs, vps;            // elements and 16-byte vectors per piece (worked out on the host: no division on the device)
-    int32_t seg_ptr_count;      // > 0: the pieces live in buffers of their own, seg_ptr[j]; 0: a stride apart in `logits`
-    int64_t seg_row_offset;     // rows to skip at the start of every piece buffer
-    const void *seg_ptr[ALBIREO_MAX_PEER_SEGMENTS];
+    int32_t nstages;            // ring depth chosen by the host for this launch
+    int32_t vps;                // 16-byte vectors per piece (worked out on the host: no division on the device)
+    int32_t Vs;                 // elements per piece
+    uint32_t flags;
+    uint32_t row_base;
     const float *temperature;
     const int32_t *top_k;
     const float *top_p, *min_p, *rep, *pres, *freq;
     const int32_t *hist_ids, *hist_off;
     const uint64_t *seeds;
+    const int32_t *out_start;   // per row: where the generated output begins in the history, or null: at 0
     uint64_t step;
-    uint32_t row_base;
-    uint32_t flags;
     int32_t *out_tokens;
     float *out_logprobs;
     int32_t num_top;
+    int32_t dbg_cap;
     int32_t *out_top_ids;
     float *out_top_logprobs;
     int32_t *out_num_kept, *out_num_topk;
-    int32_t dbg_cap;
     int32_t *dbg_topk_ids;
     uint32_t *out_row_status;
-    int32_t elem_size;          // host side only: bytes per logit
-    int32_t nstages;            // ring depth chosen by the host for this launch
-    const int32_t *out_start;   // per row: where the generated output begins in the history, or null: at 0
     const float *exp1;          // pre-generated Exp(1) variates [B, exp1_stride], or null: counter-based draw
     int64_t exp1_stride;
     int32_t *backfill_ids;      // early feedback: next iteration's input ids, or null
@@ -90,6 +88,12 @@ struct SampleArgs {
     int64_t feedback_cap, feedback_head;
     uint32_t *ws_counts;        // global scratch for history counts of rows with many distinct ids
     int64_t ws_counts_cap;      // entries
+    int32_t elem_size;          // host side only: bytes per logit
+    // rows in pieces (vocabulary shards as the all-to-all of sequence-parallel sampling leaves them)
+    int32_t seg_ptr_count;      // > 0: the pieces live in buffers of their own, seg_ptr[j]; 0: a stride apart in `logits`
+    int64_t seg_stride;         // elements between consecutive pieces of a row
+    int64_t seg_row_offset;     // rows to skip at the start of every piece buffer
+    const void *seg_ptr[ALBIREO_MAX_PEER_SEGMENTS];
 };
 
 // ------------------------------------------------------------------ scalar helpers
@@ -1279,8 +1283,12 @@ __device__ bool cand_select_pass(BlockScratch &s, const CandSmem &cs, int n, uin
     if (above < k && k <= above + mine) { s.found_digit = SEL_BINS - 1 - threadIdx.x; s.found_cnt = above; }
     __syncthreads();
     const uint32_t digit = s.found_digit;
+    const uint32_t fcnt = s.found_cnt;
+    // (everybody has the result before the next pass, or anybody else, resets it: a thread that read
+    // the reset value instead would leave the caller's loop early and miss that pass's barriers)
+    __syncthreads();
     if (digit == 0xFFFFFFFFu) return false;
-    k -= s.found_cnt;
+    k -= fcnt;
     const uint32_t nlo = lo + (digit << shift);
     uint32_t nhi = nlo + ((1u << shift) - 1u);
     if (nhi > hi || nhi < nlo) nhi = hi;
@@ -1396,6 +1404,7 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
     int rank = 0;
     if (j < n) {
         C = cs.cand[j];
+#pragma unroll 4
         for (int q = part; q < n; q += parts) rank += cs.cand[q] > C;
     }
     {
@@ -1403,8 +1412,8 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         if (t >= 0 && t < n) {
             const u64 Ct = cs.cand[t];
             nle[t] = a.exp1 ? -logf(__ldg(a.exp1 + (int64_t)b * a.exp1_stride + comp_idx(Ct)))
-                            : neg_log_exp1_f32(race_word(rp.seed, rp.R, a.step, comp_idx(Ct)));
-            mass[t] = mass_fx(__fsub_rn(unkey((uint32_t)(Ct >> 32)), zmax));
+                            : neg_log_exp1_fast(race_word(rp.seed, rp.R, a.step, comp_idx(Ct)));
+            mass[t] = mass_gen(__fsub_rn(unkey((uint32_t)(Ct >> 32)), zmax));
         }
     }
     for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
@@ -1896,6 +1905,21 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
     // stream (the producer of the logits) was still running: wait for it before anything is read or written.
     if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The launch arguments are in constant memory that no SM has seen before this launch: each 64-byte
+    // line of them costs a miss at first touch, and a warp that needs several takes them one after
+    // another.  The lines that only the end of a row needs are touched here once, each from a warp
+    // of its own, so that those misses overlap the stream instead of standing in the row's tail.
+    {
+        uint32_t touch;
+        switch (threadIdx.x >> 5) {
+            case 12: touch = (uint32_t)a.num_top + (uint32_t)a.step; break;
+            case 13: touch = (uint32_t)(uintptr_t)a.out_row_status; break;
+            case 14: touch = (uint32_t)a.backfill_len; break;
+            case 15: touch = (uint32_t)a.elem_size + (uint32_t)a.seg_row_offset; break;
+            default: touch = 1u; break;
+        }
+        if (touch == 0xFFFFFFF1u) s.bcast[3] = touch;      // (never: keeps the reads)
+    }
     const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
     if (ring_started) candidate_begin<DT>(s, rg, c);
 
