@@ -3,8 +3,8 @@
  *
  * The library implements the sampling task T4 of "Albireo" (arxiv 2606.01927, section
  * 2.1): after every decode step, for each row of the (s x v) logits matrix, choose the
- * next token.  The paper keeps "the core sampling computation" unchanged (section 6.1,
- * step 3) and enables every feature in its evaluation (section 8.1, Workload): top-p,
+ * next token.  The paper leaves the per-row sampling arithmetic as it is in the serving
+ * framework (section 6.1, step 3) and enables every feature in its evaluation (section 8.1, Workload): top-p,
  * top-k, min-p, temperature, and repetition / presence / frequency penalties driven by
  * per-sequence metadata (section 3.1, Optimization 3).  Rows are independent (section
  * 6.1), the result per row is one token id plus its probability (section 6.2, result
@@ -63,7 +63,9 @@ enum {
 #define ALBIREO_ROW_GENERAL_PATH 1u  /* informational: row took the multi-pass general path */
 #define ALBIREO_ROW_BAD_PARAM 2u     /* T < 0 or NaN, r <= 0, ...: row treated per the clamps */
 #define ALBIREO_ROW_HISTORY_OVERFLOW 4u /* history did not fit the workspace: penalties skipped */
-#define ALBIREO_ROW_TIMEOUT 8u       /* a bounded on-chip wait expired: no result for this row   */
+#define ALBIREO_ROW_TIMEOUT 8u       /* a bounded on-chip wait expired: no result for this row;
+                                        out_tokens[b] = -1 and out_logprobs[b] = NaN mark it for
+                                        callers that pass no status array                        */
 
 /* flags of albireo_sample_ext_t.flags */
 #define ALBIREO_FLAG_FORCE_GENERAL 1u /* testing: send every row down the general path     */
@@ -262,6 +264,17 @@ const char *albireo_last_error(const albireo_sampler_t *h);
 
 /* Number of kernel launches albireo_sample has enqueued through this handle so far. */
 uint64_t albireo_sample_launch_count(const albireo_sampler_t *h);
+
+/*
+ * Measurement aid (the paper has no counterpart): streams the rows of a dense [B, V] logits matrix
+ * through the sampler's own shared-memory ring, in the sampler's launch shape, testing every tile
+ * against a threshold nothing reaches -- and does nothing else.  Its duration is what the stream
+ * alone costs on this GPU at this size; benchmarks report it beside the sampler's.
+ *   sink  uint32[B] device: one word per row is written (so that the loads are kept).
+ * Asynchronous on `stream`; errors as albireo_sample.
+ */
+int albireo_stream_only(albireo_sampler_t *h, const void *logits, int32_t B, int32_t V, int32_t dtype,
+                        uint32_t *sink, void *stream);
 
 /* largest history_total albireo_sample_fixed_scratch accepts (entries of its fixed scratch array) */
 #define ALBIREO_FIXED_MAX_HISTORY (1 << 20)

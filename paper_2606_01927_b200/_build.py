@@ -43,22 +43,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
-TOOL_SRC = os.path.join(_PKG, "csrc", "read_ceiling.cu")
-TOOL_PATH = os.path.join(_PKG, "read_ceiling")
-
-
-def build_tools(force: bool = False) -> str:
-    """Compile the stand-alone read-ceiling measurement tool (see bench.py --read-ceiling)."""
-    if force or not os.path.exists(TOOL_PATH) or os.path.getmtime(TOOL_PATH) < os.path.getmtime(TOOL_SRC):
-        tmp = TOOL_PATH + f".tmp{os.getpid()}"
-        cmd = [nvcc_path(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-               "-o", tmp, TOOL_SRC]
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        if res.returncode != 0:
-            raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-        os.replace(tmp, TOOL_PATH)
-    return TOOL_PATH
-
-
 if __name__ == "__main__":
     print(build(force=True, verbose=True))

@@ -40,6 +40,7 @@ EXPORTS = [
     "albireo_sample_workspace_bytes", "albireo_sample_host_staging_bytes", "albireo_sample_init",
     "albireo_sample", "albireo_sample_host", "albireo_sample_destroy", "albireo_last_error",
     "albireo_sample_launch_count", "albireo_sample_fixed_scratch", "albireo_sample_fixed_scratch_error",
+    "albireo_stream_only",
 ]
 
 
@@ -91,6 +92,8 @@ def _load() -> C.CDLL:
     lib.albireo_sample_fixed_scratch.argtypes = sample_args[1:14] + [i64] + sample_args[14:]
     lib.albireo_sample_fixed_scratch_error.restype = C.c_char_p
     lib.albireo_sample_fixed_scratch_error.argtypes = []
+    lib.albireo_stream_only.restype = C.c_int
+    lib.albireo_stream_only.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     return lib
 
 
@@ -288,6 +291,18 @@ class Sampler:
         if rc != OK:
             raise AlbireoError(rc, self.last_error())
         return SampleOutputs(out_tokens, out_logprobs, **extra)
+
+    def albireo_stream_only(self, logits: torch.Tensor, sink: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+        """Measurement aid: the sampler's stream over ``logits`` ([B, V], dense) and nothing else."""
+        B, V = logits.shape
+        if not logits.is_contiguous() or sink.dtype != torch.int32 or sink.numel() < B:
+            raise ValueError("albireo_stream_only wants dense logits and an int32 sink of B words")
+        st = torch.cuda.current_stream(logits.device) if stream is None else stream
+        with torch.cuda.device(logits.device):
+            rc = LIB.albireo_stream_only(self._handle, C.c_void_p(logits.data_ptr()), B, V, _dtype_code(logits),
+                                         C.c_void_p(sink.data_ptr()), C.c_void_p(st.cuda_stream))
+        if rc != OK:
+            raise AlbireoError(rc, self.last_error())
 
     def albireo_sample_host(self, logits: torch.Tensor, *, temperature=None, top_k=None, top_p=None, min_p=None,
                             repetition_penalty=None, presence_penalty=None, frequency_penalty=None,

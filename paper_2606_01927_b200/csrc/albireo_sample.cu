@@ -609,7 +609,7 @@ __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, co
     uint32_t *cnt;
     bool ok = true;
     if (U <= CNT_CAP) cnt = hs.counts;
-    else if (ws && ws_off + (int64_t)U <= ws_cap) cnt = ws + ws_off;
+    else if (ws && ws_off >= 0 && ws_off + (int64_t)U <= ws_cap) cnt = ws + ws_off;
     else { cnt = nullptr; ok = false; }
     c.bitmap = hs.bitmap; c.coarse = hs.coarse; c.counts = cnt; c.n_distinct = U; c.ncoarse = ncoarse;
     if (!ok) return false;
@@ -1679,7 +1679,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
             if (threadIdx.x == 0 && (uint32_t)tile == s.maint_at) s.maint_at = 0xFFFFFFFFu;
             if (ovf || tmo) {
                 ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
-                if (tmo) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; return true; }
+                if (tmo) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); out.n_keep = 0; out.n_topk = 0; return true; }
                 __syncthreads();
                 return false;
             }
@@ -1799,7 +1799,7 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     __syncthreads();
     if (s.timeout) {
         ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
-        out.status |= ALBIREO_ROW_TIMEOUT; out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0;
+        out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); out.n_keep = 0; out.n_topk = 0;
         return true;
     }
     // scalar head and tail of a row that is not 16-byte aligned / not a whole number of vectors
@@ -1986,7 +1986,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
         // (the barrier above made s.issued visible)
         bool landed = mbar_wait(&rg.bar[MAX_STAGES - 1], 0u);
         for (int t = 0; t < (int)s.issued; ++t) landed = mbar_wait(&rg.bar[t], 0u) && landed;
-        if (__syncthreads_or(!landed)) { out.status |= ALBIREO_ROW_TIMEOUT; done = true; }   // the same in every thread
+        if (__syncthreads_or(!landed)) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); done = true; }   // the same in every thread
     }
     if (!done) {
         __syncthreads();
@@ -2015,6 +2015,76 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
         }
         if (a.out_row_status) a.out_row_status[b] = out.status;
     }
+}
+
+// ------------------------------------------------------------------ the stream alone (measurement aid)
+//
+// The same ring, the same launch shape (a CTA per row, 512 threads, two CTAs per SM), the same
+// packed test of every tile against a threshold nothing reaches -- and nothing else: no threshold to
+// set up, no candidates, no final stage.  What this kernel takes is what the stream itself costs on
+// this GPU at this size; the sampler's own work is the difference.  Writes one word per row so that
+// the loads cannot be dropped.
+template <int DT>
+__global__ void __launch_bounds__(NT, 2) albireo_stream_only_kernel(const void *logits, int V, int64_t row_stride, int nstages, uint32_t *sink) {
+    typedef Elem<DT> E;
+    typedef VecTest<DT> T;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ uint32_t done[MAX_STAGES];
+    __shared__ uint32_t hits, dead;
+    __shared__ const char *no_pieces[1];
+    Ring rg;
+    rg.nstages = nstages; rg.vps = 0x7FFFFFFF; rg.seg_base = no_pieces;
+    rg.buf = smem + COMMON_BYTES;
+    rg.bar = (uint64_t *)(rg.buf + (size_t)nstages * STAGE_BYTES);
+    const char *row = (const char *)logits + (size_t)blockIdx.x * (size_t)row_stride * E::SIZE;
+    int head = (int)(((16u - (uint32_t)((uintptr_t)row & 15u)) & 15u) / E::SIZE);
+    if (head > V) head = V;
+    const int nvec = (V - head) / E::PER_VEC;
+    const uint4 *vp = (const uint4 *)(row + (size_t)head * E::SIZE);
+    const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
+    if (threadIdx.x == 0) {
+        for (int st = 0; st < nstages; ++st) { mbar_init(&rg.bar[st], 1); done[st] = 0; }
+        hits = 0; dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const int npre = ntiles < nstages ? ntiles : nstages;
+        for (int t = 0; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int pvec = 16 * lane + (((threadIdx.x >> 5) + lane) & 15);
+    const uint32_t thr = T::raw_threshold(KEY_POS_INF - 1u, 1.0f);
+    int st = 0; uint32_t parity = 0, cnt = 0;
+    for (int tile = 0; tile < ntiles; ++tile) {
+        if (*(volatile uint32_t *)&dead == 0u) {
+            if (!mbar_wait(&rg.bar[st], parity)) dead = 1u;        // (bounded: the row is given up, the protocol below goes on)
+            else {
+                const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + pvec;
+                const int vbase = tile * NT * TILE_VECS;
+                uint4 cur[TILE_VECS];
+#pragma unroll
+                for (int u = 0; u < TILE_VECS; ++u) cur[u] = (vbase + u * NT + pvec < nvec) ? stage[u * NT] : T::fill();
+                if (__any_sync(0xFFFFFFFFu, T::any_may_pass(cur, thr, 1.0f))) cnt += 1;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence_block();
+            const uint32_t old = atomicAdd(&done[st], 1u);
+            if (old == (uint32_t)(NWARPS - 1)) {
+                done[st] = 0;
+                __threadfence_block();
+                if (tile + nstages < ntiles && *(volatile uint32_t *)&dead == 0u) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    ring_issue(rg, vp, nvec, tile + nstages, st);
+                }
+            }
+        }
+        if (++st == nstages) { st = 0; parity ^= 1u; }
+    }
+    if (cnt && lane == 0) atomicAdd(&hits, cnt);
+    __syncthreads();
+    if (threadIdx.x == 0) sink[blockIdx.x] = hits + (dead << 31);
 }
 
 size_t history_smem_bytes(int V) {
@@ -2133,6 +2203,9 @@ size_t enable_large_smem(int device, cudaError_t *err) {
     e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_sample_kernel<ALBIREO_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_stream_only_kernel<ALBIREO_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_stream_only_kernel<ALBIREO_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(albireo_stream_only_kernel<ALBIREO_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     *err = e;
     return e == cudaSuccess ? smem : 0;
 }
@@ -2272,6 +2345,7 @@ extern "C" int albireo_sample_host(albireo_sampler_t *h, const void *logits, int
     if (ext && ext->struct_size != sizeof(albireo_sample_ext_t)) { set_err(h, "ext->struct_size mismatch%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->row_stride_elems != 0 && ext->row_stride_elems != V) { set_err(h, "host entry needs dense rows%s", ""); return ALBIREO_EINVAL; }
     if (ext && ext->dbg_cap > 0) { set_err(h, "host entry has no debug output%s", ""); return ALBIREO_EINVAL; }
+    if (ext && (ext->num_top < 0 || ext->num_top > ALBIREO_MAX_NUM_TOP)) { set_err(h, "num_top out of range%s", ""); return ALBIREO_EUNSUPPORTED; }
     if (ext && (ext->exp1 || ext->backfill_ids || ext->feedback_ring || ext->num_segments > 1 || ext->history_output_start)) { set_err(h, "host entry takes no exp1 table, no early-feedback targets, no rows in pieces and no history split%s", ""); return ALBIREO_EINVAL; }
     const size_t base = albireo_sample_workspace_bytes(h->max_rows, h->max_vocab, h->max_history_total);
     if (h->workspace_bytes < base + albireo_sample_host_staging_bytes(h->max_rows, h->max_vocab, h->max_history_total)) {
@@ -2309,7 +2383,6 @@ extern "C" int albireo_sample_host(albireo_sampler_t *h, const void *logits, int
     dx.struct_size = sizeof dx;
     if (ext) {
         dx.flags = ext->flags; dx.row_base = ext->row_base; dx.num_top = ext->num_top;
-        if (ext->num_top < 0 || ext->num_top > ALBIREO_MAX_NUM_TOP) { set_err(h, "num_top out of range%s", ""); return ALBIREO_EUNSUPPORTED; }
         if (ext->out_num_kept) dx.out_num_kept = (int32_t *)reserve(Bs * 4);
         if (ext->out_num_topk) dx.out_num_topk = (int32_t *)reserve(Bs * 4);
         if (ext->out_row_status) dx.out_row_status = (uint32_t *)reserve(Bs * 4);
@@ -2349,6 +2422,26 @@ extern "C" int albireo_sample_destroy(albireo_sampler_t *h) {
 extern "C" const char *albireo_last_error(const albireo_sampler_t *h) { return h ? h->err : ""; }
 
 extern "C" uint64_t albireo_sample_launch_count(const albireo_sampler_t *h) { return h ? h->launches : 0; }
+
+// Launches albireo_stream_only_kernel on the rows of `logits` (dense [B, V], one piece per row): see there.
+extern "C" int albireo_stream_only(albireo_sampler_t *h, const void *logits, int32_t B, int32_t V, int32_t dtype,
+                                   uint32_t *sink, void *stream) {
+    if (!h) return ALBIREO_EINVAL;
+    h->err[0] = 0;
+    if (B == 0) return ALBIREO_OK;
+    if (B < 0 || B > h->max_rows || V < 1 || V > h->max_vocab || !logits || !sink) { set_err(h, "bad arguments%s", ""); return ALBIREO_EINVAL; }
+    if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16 && dtype != ALBIREO_F16) { set_err(h, "unknown dtype%s", ""); return ALBIREO_EINVAL; }
+    const int nstages = ring_stages_for(V, false);
+    const size_t smem = smem_bytes_for(V, false, nstages);
+    if (smem > h->max_smem) { set_err(h, "vocabulary too large%s", ""); return ALBIREO_EUNSUPPORTED; }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == ALBIREO_F32) albireo_stream_only_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
+    else if (dtype == ALBIREO_BF16) albireo_stream_only_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
+    else albireo_stream_only_kernel<ALBIREO_F16><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_err(h, "kernel launch failed: %s", cudaGetErrorString(e)); return ALBIREO_ECUDA; }
+    return ALBIREO_OK;
+}
 
 // ------------------------------------------------------------------ entry point that allocates nothing
 //
