@@ -7,7 +7,9 @@ module.  It shares no code with the CUDA library; the product never routes throu
 enumerates, for one row, every (token, logprob) pair the definition yields when the
 two real-valued cut parameters are moved inside their backward-error bands
 (ln(min_p) by <= 1e-5, top_p by <= 1e-6) and, where the two best race scores are
-closer than 1e-5, the runner-up token as well.
+closer than 1e-5 x max(1, their magnitude), the runner-up token as well.  In the
+full-vocabulary log-probability mode every enumerated log-probability is relative to the
+whole row, as the primary result's is.
 """
 from __future__ import annotations
 
@@ -212,7 +214,7 @@ def acceptable(w, b: int):
 
     The first entry is the primary result.  The rest come from moving ln(min_p) within
     +-1e-5 and top_p within +-1e-6 (every kept-prefix length reachable inside the
-    bands), and from near-ties of the race (gap < 1e-5 between the two best scores).
+    bands), and from near-ties of the race (gap < 1e-5 x max(1, |score|) between the two best scores).
     """
     prim, ids, zs, gs = row_shifted(w, b, 0.0, 0.0, want_sorted=True)
     out = [(int(prim["token"]), float(prim["logprob"]), int(prim["n_keep"]))]
@@ -236,6 +238,14 @@ def acceptable(w, b: int):
     else:
         L7s = [L6]
 
+    # the full-vocabulary mode measures probabilities against every finite score of the row
+    full = bool(getattr(w, "logprob_full_vocab", False))
+    S_full = float(np.sum(np.exp(d[np.isfinite(d)]))) if full else None
+
+    def near_tie(ga, gb):
+        # race scores are differences of O(1..100) terms: the band scales with their size
+        return ga - gb < RACE_BAND * max(1.0, abs(ga), abs(gb))
+
     seen = set()
     for L7 in L7s:
         e = np.exp(d[:L7])
@@ -257,12 +267,12 @@ def acceptable(w, b: int):
                 continue
             seen.add(L8)
             g = gs[:L8]
-            S = float(np.sum(e[:L8]))
+            S = S_full if full else float(np.sum(e[:L8]))
             order = np.lexsort((ids[:L8], -g))       # best g first, ties -> lowest id
             jb = int(order[0])
             out.append((int(ids[jb]), float(d[jb] - np.log(S)), L8))
             if L8 > 1:
                 j2 = int(order[1])
-                if g[jb] - g[j2] < RACE_BAND:
+                if near_tie(float(g[jb]), float(g[j2])):
                     out.append((int(ids[j2]), float(d[j2] - np.log(S)), L8))
     return out

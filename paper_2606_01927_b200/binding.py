@@ -340,10 +340,12 @@ def albireo_sample_fixed_scratch(logits: torch.Tensor, *, temperature=None, top_
                                  repetition_penalty=None, presence_penalty=None, frequency_penalty=None,
                                  history_ids=None, history_offsets=None, history_total: Optional[int] = None,
                                  seeds=None, step: int = 0, out_tokens=None, out_logprobs=None,
-                                 stream: Optional[torch.cuda.Stream] = None, row_base: int = 0) -> SampleOutputs:
+                                 stream: Optional[torch.cuda.Stream] = None, row_base: int = 0,
+                                 want_status: bool = False, want_counts: bool = False) -> SampleOutputs:
     """The sampler for callers that may not allocate: no handle, no workspace (the library's own
-    fixed scratch array is used).  The output tensors created here when none are passed are a
-    convenience of this Python wrapper; the C entry point itself allocates nothing."""
+    fixed scratch array is used).  The output tensors created here when none are passed (and the
+    per-row status / count arrays when asked for) are a convenience of this Python wrapper; the C
+    entry point itself allocates nothing."""
     B, V = logits.shape
     dt = _dtype_code(logits)
     dev = logits.device
@@ -354,6 +356,14 @@ def albireo_sample_fixed_scratch(logits: torch.Tensor, *, temperature=None, top_
     ext = SampleExt()
     ext.struct_size = C.sizeof(SampleExt)
     ext.row_base = row_base
+    row_status = num_kept = num_topk = None
+    if want_status:
+        row_status = torch.zeros(B, dtype=torch.int32, device=dev)
+        ext.out_row_status = row_status.data_ptr()
+    if want_counts:
+        num_kept = torch.empty(B, dtype=torch.int32, device=dev)
+        num_topk = torch.empty(B, dtype=torch.int32, device=dev)
+        ext.out_num_kept, ext.out_num_topk = num_kept.data_ptr(), num_topk.data_ptr()
     if history_total is None:
         history_total = int(history_ids.numel()) if history_ids is not None else 0
     st = torch.cuda.current_stream(dev) if stream is None else stream
@@ -369,7 +379,7 @@ def albireo_sample_fixed_scratch(logits: torch.Tensor, *, temperature=None, top_
             C.c_void_p(st.cuda_stream), C.byref(ext))
     if rc != OK:
         raise AlbireoError(rc, LIB.albireo_sample_fixed_scratch_error().decode())
-    return SampleOutputs(out_tokens, out_logprobs)
+    return SampleOutputs(out_tokens, out_logprobs, num_kept=num_kept, num_topk=num_topk, row_status=row_status)
 
 
 # ------------------------------------------------------------------ workload marshalling

@@ -8,10 +8,11 @@ Rules (tolerances written out here, nowhere else):
     debug capacity;
   * logprob: |gpu - oracle| <= LOGPROB_TOL (absolute) against the primary result; the output is an
     fp32, whose spacing exceeds that once |logprob| passes about 170 (probabilities below e^-170,
-    met only in top-N lists at tiny temperatures), so two fp32 spacings of the value are allowed on top;
+    met only in top-N lists at tiny temperatures), so two fp32 spacings of the value are allowed on top
+    where that spacing is above 1e-6 (|logprob| >= 16); below that the bound is the plain 2e-5;
   * token: identical to the primary result, except *excused* rows: the GPU's
     (token, logprob) matches one of the results the definition gives when ln(min_p) moves
-    by <= 1e-5, top_p by <= 1e-6, or the two best race scores are closer than 1e-5.
+    by <= 1e-5, top_p by <= 1e-6, or the two best race scores are closer than 1e-5 x max(1, |score|).
     Excused rows are counted; unexcused mismatches must be zero.
 The final kept-set size is diagnostic only (it is ill-conditioned for diffuse rows).
 """
@@ -24,11 +25,17 @@ import numpy as np
 from oracle import albireo_oracle as O
 
 LOGPROB_TOL = 2e-5
+# the fp32 output's own spacing is added to the tolerance only where it is no longer negligible
+# beside LOGPROB_TOL (|logprob| >= 16: spacing 1.9e-6); ordinary values get the plain 2e-5
+FP32_SPACING_FLOOR = 1e-6
 
 
 def logprob_tol(ref):
     """Allowed |gpu - oracle| for a log-probability whose oracle value is ``ref``."""
-    return LOGPROB_TOL + 2.0 * np.spacing(np.abs(np.asarray(ref, dtype=np.float64)).astype(np.float32)).astype(np.float64)
+    sp = np.spacing(np.abs(np.asarray(ref, dtype=np.float64)).astype(np.float32)).astype(np.float64)
+    return LOGPROB_TOL + np.where(sp > FP32_SPACING_FLOOR, 2.0 * sp, 0.0)
+
+
 EXCUSED_FRACTION = 1e-3
 
 

@@ -73,7 +73,7 @@ SMALL = [
 def test_small_mixed_parameters(binding, sampler, seed, B, V, dtype, q, flags):
     w = W.random_small(seed, B=B, V=V, dtype=dtype, quantise=q)
     w.num_top = 5
-    check(binding, sampler, w, flags=flags, allow_excused=1)
+    check(binding, sampler, w, flags=flags, allow_excused=0)
 
 
 @pytest.mark.parametrize("flags", [0, 1], ids=["auto", "general"])
@@ -82,7 +82,7 @@ def test_small_no_history_no_arrays(binding, sampler, flags):
     rng = np.random.default_rng(5)
     x = (rng.standard_normal((24, 5000)) * 2).astype(np.float32)
     w = W.Workload("plain", 24, 5000, W.BF16, W.f32_to_bf16_bits(x))
-    check(binding, sampler, w, flags=flags, allow_excused=1)
+    check(binding, sampler, w, flags=flags, allow_excused=0)
 
 
 # ------------------------------------------------------------------ degenerate rows
@@ -120,10 +120,15 @@ def test_degenerate_rows(binding, sampler, dtype, flags):
         dict(temperature=np.full(n, 1.0, np.float32), top_k=np.full(n, 300, np.int32), min_p=np.full(n, 1.5, np.float32)),
         dict(temperature=np.full(n, 1.0, np.float32), top_p=np.zeros(n, np.float32)),
     ]
+    excused = 0
     for i, kw in enumerate(variants):
         w = W.Workload(f"degenerate{i}", n, V, dtype, x if dtype == W.F32 else W.f32_to_bf16_bits(x),
                        seeds=np.arange(n, dtype=np.uint64) + 11, step=3, num_top=8, **kw)
-        check(binding, sampler, w, flags=flags, allow_excused=1)
+        rep, _ = check(binding, sampler, w, flags=flags, allow_excused=1)
+        excused += len(rep.excused)
+    # flat rows put thousands of equal masses at the top-p cut, so a row inside the cut's error band can
+    # occur; over the 72 rows of the eight variants no more than one may
+    assert excused <= 1, excused
 
 
 def test_history_with_many_distinct_ids_uses_workspace(binding, sampler):

@@ -659,3 +659,140 @@ def test_full_vocabulary_logprobs_equal_library_log_softmax_whatever_the_cuts():
     ref0 = scipy.special.log_softmax(x.astype(np.float64), axis=1)
     for b in range(B):
         assert og.tokens[b] == int(np.argmax(x[b])) and abs(og.logprobs[b] - ref0[b, og.tokens[b]]) < 1e-12
+
+
+# ------------------------------------------------------------------ race ties, out-of-contract parameters, band enumeration
+
+def test_race_tie_goes_to_the_lowest_id():
+    # equal scores and equal variates give equal race scores g: the lowest id of the tied best wins,
+    # wherever the tied ids sit in the sorted order and whatever id carries the (lower) rest
+    V = 40
+    x = np.full((3, V), -3.0, dtype=np.float32)
+    tied = [[7, 19, 33], [0, 39], [38, 5, 21, 6]]
+    for b, ids in enumerate(tied):
+        x[b, ids] = 2.0
+    w = one_row(x, T=1.0, seed=9)
+    E = np.full((3, V), 0.75, dtype=np.float32)
+    w.exp1 = E.copy()
+    o = O.sample(w)
+    assert o.tokens.tolist() == [min(t) for t in tied]
+    assert (o.rows["race_gap"] == 0.0).all()
+    # equal g from unequal parts: z lower by ln 2 exactly where E is halved (z = k ln 2 is not exact in fp32,
+    # so build it the other way round: E' = E * exp(z' - z) in fp64, rounded once -- the tie is then only
+    # near, and the winner is whichever g is larger, computed here from the same fp32 inputs)
+    x2 = np.full((1, V), -30.0, dtype=np.float32)
+    x2[0, [4, 9]] = [1.0, 0.5]
+    w2 = one_row(x2, T=1.0, seed=9)
+    E2 = np.full((1, V), 0.5, dtype=np.float32)
+    E2[0, 9] = np.float32(0.5 * math.exp(-0.5))
+    w2.exp1 = E2
+    g4 = (1.0 - 1.0) - math.log(float(E2[0, 4]))
+    g9 = (0.5 - 1.0) - math.log(float(E2[0, 9]))
+    want = 4 if (g4 > g9 or (g4 == g9)) else 9
+    assert O.sample(w2).tokens[0] == want
+    # the tie rule does not depend on the cut that built the kept set
+    w3 = one_row(x, T=1.0, top_k=2, seed=9)
+    w3.exp1 = E.copy()
+    assert O.sample(w3).tokens.tolist() == [7, 0, 5]
+
+
+def test_negative_and_nan_temperature_mean_greedy():
+    # T <= 0 is greedy; the same reading covers a negative and a NaN temperature (anything not > 0)
+    rng = np.random.default_rng(71)
+    x = (rng.standard_normal((6, 500)) * 3).astype(np.float32)
+    x[2, [17, 300]] = x[2].max() + 1.0                      # a tie at the top: lowest id
+    ref = O.sample(one_row(x, T=0.0, top_k=40, top_p=0.5, min_p=0.2, seed=3))
+    for T in (-1.0, -np.inf, np.nan, -0.0):
+        o = O.sample(one_row(x, T=T, top_k=40, top_p=0.5, min_p=0.2, seed=3))
+        assert (o.rows["greedy"] == 1).all()
+        assert o.tokens.tolist() == [int(np.argmax(r)) for r in x] == ref.tokens.tolist()
+        assert (o.logprobs == 0.0).all() and (o.rows["n_keep"] == 1).all()
+    assert ref.tokens[2] == 17
+
+
+def test_nonpositive_repetition_penalty_is_plain_arithmetic():
+    # r <= 0 is outside the method's contract; the definition is applied as written (x / r for x > 0,
+    # x * r otherwise), one fp32 rounding per operation, so that both implementations agree on such rows
+    rng = np.random.default_rng(72)
+    V = 64
+    x = (rng.standard_normal(V) * 3).astype(np.float32)
+    hist = [3, 3, 10, 40, 63]
+    for r in (-1.5, -0.25):
+        z = O.row_scores(x, W.F32, T=1.0, r=r, history=hist)
+        want = x.copy()
+        for t in set(hist):
+            want[t] = np.float32(x[t] / np.float32(r)) if x[t] > 0 else np.float32(x[t] * np.float32(r))
+        assert (z.view(np.uint32) == want.view(np.uint32)).all()
+        w = one_row(x[None], T=1.0, r=r, history=hist, top_k=5, seed=2)
+        o = O.sample(w, kept_cap=5)
+        order = np.lexsort((np.arange(V), -want.astype(np.float64)))
+        assert o.kept_ids[0].tolist() == order[:5].tolist()
+
+
+def test_shifted_cut_parameters_equal_changed_parameters():
+    # the oracle's "same row, cut parameter moved" entry against the plain entry with the moved parameter
+    # itself, for moves that are exact in fp32 (top_p 0.75 -> 0.5 and 0.25 -> 0.5; min_p 0.125 -> 0.25)
+    rng = np.random.default_rng(73)
+    x = (rng.standard_normal((8, 300)) * 2).astype(np.float32)
+    for p0, dp in ((0.75, -0.25), (0.25, 0.25)):
+        a = one_row(x, T=1.0, top_p=p0, seed=4)
+        b = O.sample(one_row(x, T=1.0, top_p=p0 + dp, seed=4))
+        for i in range(8):
+            r, _, _, _ = O.row_shifted(a, i, 0.0, dp)
+            assert (r["token"], r["n_keep"]) == (b.tokens[i], b.rows["n_keep"][i])
+            assert r["logprob"] == b.logprobs[i]
+    a = one_row(x, T=1.0, min_p=0.125, seed=4)
+    b = O.sample(one_row(x, T=1.0, min_p=0.25, seed=4))
+    for i in range(8):
+        r, _, _, _ = O.row_shifted(a, i, math.log(2.0), 0.0)
+        assert (r["token"], r["n_keep"]) == (b.tokens[i], b.rows["n_keep"][i])
+    assert (b.rows["n_keep"] < O.sample(a).rows["n_keep"]).any()        # (the move does change the cut)
+
+
+def test_band_enumeration_contains_every_shifted_result():
+    # acceptable() enumerates the kept-prefix lengths reachable inside the bands with numpy; every result of
+    # the C entry with the parameters moved to the ends (and the middle) of the bands must be among them,
+    # in the ordinary and in the full-vocabulary log-probability mode
+    rng = np.random.default_rng(74)
+    x = np.round(rng.standard_normal((6, 400)) * 2, 1).astype(np.float32)        # many exact ties
+    x[0] = 0.0                                                                    # flat row: cut on a boundary
+    for full in (False, True):
+        for kw in (dict(top_p=0.5), dict(min_p=float(np.exp(np.float32(-1.0)))), dict(top_p=0.9, min_p=0.05, top_k=50)):
+            w = one_row(x, T=1.0, seed=6, **kw)
+            w.logprob_full_vocab = full
+            for b in range(6):
+                acc = O.acceptable(w, b)
+                prim, _, _, _ = O.row_shifted(w, b, 0.0, 0.0)
+                assert (acc[0][0], acc[0][2]) == (prim["token"], prim["n_keep"]) and acc[0][1] == prim["logprob"]
+                for s7 in (-O.LN_MIN_P_BAND, 0.0, O.LN_MIN_P_BAND):
+                    for s8 in (-O.TOP_P_BAND, 0.0, O.TOP_P_BAND):
+                        r, _, _, _ = O.row_shifted(w, b, s7 * 0.999, s8 * 0.999)
+                        assert any(t == r["token"] and n == r["n_keep"] and abs(lp - r["logprob"]) < 1e-12
+                                   for (t, lp, n) in acc), (full, kw, b, s7, s8)
+    # full-vocabulary mode: the enumerated log-probabilities are relative to the whole row
+    w = one_row(x, T=1.0, seed=6, top_p=0.5)
+    w.logprob_full_vocab = True
+    ls = scipy.special.log_softmax(x.astype(np.float64), axis=1)
+    for b in range(6):
+        for (t, lp, _) in O.acceptable(w, b):
+            assert abs(lp - ls[b, t]) < 1e-12
+
+
+def test_race_near_tie_band_is_relative():
+    # two survivors whose race scores differ by 3e-5 at |g| ~ 20: inside the relative band (1e-5 * 20),
+    # so the runner-up is acceptable; the same gap at |g| ~ 1 is outside it
+    def two(z1, e0, e1):
+        x = np.full((1, 8), -200.0, dtype=np.float32)
+        x[0, 0], x[0, 1] = 0.0, z1
+        w = one_row(x, T=1.0, top_k=2, seed=1)
+        E = np.ones((1, 8), dtype=np.float32)
+        E[0, 0], E[0, 1] = e0, e1
+        w.exp1 = E
+        return w
+    w = two(0.0, math.exp(-20.0), math.exp(-20.0 + 3e-5))
+    gap = O.sample(w).rows["race_gap"][0]
+    assert 1e-5 < gap < 1e-4
+    assert {a[0] for a in O.acceptable(w, 0)} == {0, 1}
+    w = two(0.0, math.exp(-1.0), math.exp(-1.0 + 3e-5))
+    assert 1e-5 < O.sample(w).rows["race_gap"][0] < 1e-4
+    assert {a[0] for a in O.acceptable(w, 0)} == {0}

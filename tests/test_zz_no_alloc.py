@@ -6,8 +6,10 @@ queued around the call, or their process forbids allocation after start-up.  The
 provide the workspace that `albireo_sample_init` asks for, so `albireo_sample_fixed_scratch`
 keeps its only scratch (history occurrence counts for rows with very many distinct ids) in
 a fixed array inside the library.  This test drives that entry point through the C ABI on
-rows that really use the scratch and checks it against the ordinary entry point, twice in
-a row, because the array is shared and keeps the previous call's contents.
+rows that really use the scratch and checks it against the CPU oracle (the rules of the parity
+tests) and against the ordinary entry point (bit for bit), twice in a row, because the array is
+shared and keeps the previous call's contents; the per-row status must show no overflow of the
+history counts and no other fault.
 
 The file name makes pytest collect it last, so a run that stops at the first failure has
 already run everything else.
@@ -16,11 +18,12 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import albireo_oracle as O
 from paper_2606_01927_b200 import workloads as W
 
-pytestmark = pytest.mark.gpu
+from parity import compare, to_host
 
-LOGPROB_TOL = 2e-5      # the tolerance of the parity tests
+pytestmark = pytest.mark.gpu
 
 
 def _workload(seed, B=6, V=30000):
@@ -49,14 +52,22 @@ def test_fixed_scratch_entry_matches_the_workspace_entry_twice_in_a_row():
         w = _workload(seed)
         t = binding.workload_tensors(w, dev)
         logits = t.pop("logits")
-        got = binding.albireo_sample_fixed_scratch(logits, **t)
+        got = binding.albireo_sample_fixed_scratch(logits, **t, want_status=True, want_counts=True)
         sampler = binding.Sampler(max_rows=w.B, max_vocab=w.V, max_history_total=int(w.history_ids.size), device=dev)
-        ref = sampler.albireo_sample(logits, **t, want_status=True)
+        ref = sampler.albireo_sample(logits, **t, want_status=True, want_counts=True)
         torch.cuda.synchronize()
-        assert not (ref.row_status.cpu().numpy() & binding.ROW_HISTORY_OVERFLOW).any()
+        # the per-row status: nothing but the path bit may be set (no history overflow, no timeout, ...)
+        bad_bits = ~np.int32(binding.ROW_GENERAL_PATH)
+        assert not (got.row_status.cpu().numpy() & bad_bits).any(), (call, got.row_status.cpu().numpy())
+        assert not (ref.row_status.cpu().numpy() & bad_bits).any()
+        # against the CPU oracle, by the rules of the parity tests
+        rep = compare(w, to_host(got), O.sample(w, threads=4))
+        print(rep.summary())
+        assert rep.ok() and not rep.excused, (call, rep.failures[:3], rep.excused[:3])
+        # and against the entry point with a workspace: the same kernel, so the same bits
         assert (got.tokens.cpu().numpy() == ref.tokens.cpu().numpy()).all(), call
-        d = np.abs(got.logprobs.cpu().numpy().astype(np.float64) - ref.logprobs.cpu().numpy().astype(np.float64))
-        assert d.max() <= LOGPROB_TOL, (call, d.max())
+        assert (got.logprobs.cpu().numpy().view(np.uint32) == ref.logprobs.cpu().numpy().view(np.uint32)).all(), call
+        assert (got.num_kept.cpu().numpy() == ref.num_kept.cpu().numpy()).all(), call
         sampler.close()
 
 
