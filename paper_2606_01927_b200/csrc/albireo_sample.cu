@@ -571,25 +571,48 @@ __device__ uint32_t block_exscan_u32(BlockScratch &s, uint32_t v, uint32_t &tota
     return base + inc - v;
 }
 
-// Builds the per-row penalty tables.  Returns false (penalties skipped) if the distinct
-// ids fit neither on chip nor in the caller's workspace.
+// The first HIST_STAGED ids of a row's history are copied into shared memory at the very start of the
+// row (asynchronous 4-byte copies, no registers held, by the threads after warp 0, which is busy
+// starting the ring): the two sweeps over the ids then read them from there.  What is left of a
+// longer history is re-read from global memory.  The staging area is the candidate list, which
+// nothing uses before the stream begins.
+constexpr int HIST_STAGED = CAND_CAP * 2;      // 8 KiB of ids
+constexpr int HIST_HOLDERS = NT - 32;
+__device__ __forceinline__ void hist_prefetch(const int32_t *ids, int len, int32_t *staged) {
+    if (threadIdx.x < 32) return;
+    const int n = len < HIST_STAGED ? len : HIST_STAGED;
+    for (int j = (int)threadIdx.x - 32; j < n; j += HIST_HOLDERS)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(staged + j)), "l"(ids + j) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// Builds the per-row penalty tables from the staged ids (see hist_prefetch) and, for a longer
+// history, the rest of `ids`.  Returns false (penalties skipped) if the distinct ids fit neither on
+// chip nor in the caller's workspace.
 // Ids before position out_start are the prompt: they set their bit (repetition penalty) but are not counted.
+// Histories repeat a few ids very often: a bit already set is not set again.  (Combining equal ids
+// within a warp first, with match.any, was measured and cost far more than the atomics it saved.)
 __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, const int32_t *ids, int len, int out_start,
-                              uint32_t *ws, int64_t ws_cap, int64_t ws_off) {
+                              const int32_t *staged, uint32_t *ws, int64_t ws_cap, int64_t ws_off) {
     const int V = c.V;
     const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
-    // the first 8 ids of every thread stay in registers for the second sweep
-    constexpr int KEEP = 8;
-    int mine[KEEP];
-#pragma unroll
-    for (int q = 0; q < KEEP; ++q) { const int j = threadIdx.x + q * NT; mine[q] = j < len ? __ldg(ids + j) : -1; }
+    const int nst = len < HIST_STAGED ? len : HIST_STAGED;
     for (int w = threadIdx.x; w <= nwords; w += NT) hs.bitmap[w] = 0;
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
-#pragma unroll
-    for (int q = 0; q < KEEP; ++q) { const int t = mine[q]; if (t >= 0 && t < V) atomicOr(&hs.bitmap[t >> 5], 1u << (t & 31)); }
-    for (int j = threadIdx.x + KEEP * NT; j < len; j += NT) {
-        int t = __ldg(ids + j);
-        if (t >= 0 && t < V) atomicOr(&hs.bitmap[t >> 5], 1u << (t & 31));
+    for (int j = threadIdx.x; j < nst; j += NT) {
+        const int t = staged[j];
+        if (t >= 0 && t < V) {
+            const uint32_t bit = 1u << (t & 31);
+            if (!(*(volatile uint32_t *)&hs.bitmap[t >> 5] & bit)) atomicOr(&hs.bitmap[t >> 5], bit);
+        }
+    }
+    for (int j = threadIdx.x + HIST_STAGED; j < len; j += NT) {
+        const int t = __ldg(ids + j);
+        if (t >= 0 && t < V) {
+            const uint32_t bit = 1u << (t & 31);
+            if (!(*(volatile uint32_t *)&hs.bitmap[t >> 5] & bit)) atomicOr(&hs.bitmap[t >> 5], bit);
+        }
     }
     __syncthreads();
     // coarse exclusive prefix: one entry per 8 words; ncoarse <= 2048 for V <= 2^19
@@ -598,7 +621,12 @@ __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, co
         int cb = base + threadIdx.x;
         uint32_t pc = 0;
         if (cb < ncoarse) {
-            for (int w = cb << 3; w < min(nwords, (cb << 3) + 8); ++w) pc += __popc(hs.bitmap[w]);
+            if ((cb << 3) + 8 <= nwords) {
+                const uint4 w0 = *(const uint4 *)&hs.bitmap[cb << 3], w1 = *(const uint4 *)&hs.bitmap[(cb << 3) + 4];
+                pc = __popc(w0.x) + __popc(w0.y) + __popc(w0.z) + __popc(w0.w) + __popc(w1.x) + __popc(w1.y) + __popc(w1.z) + __popc(w1.w);
+            } else {
+                for (int w = cb << 3; w < nwords; ++w) pc += __popc(hs.bitmap[w]);
+            }
         }
         uint32_t tot;
         uint32_t ex = block_exscan_u32(s, pc, tot);
@@ -615,9 +643,11 @@ __device__ bool build_history(BlockScratch &s, const HistSmem &hs, RowCtx &c, co
     if (!ok) return false;
     for (uint32_t u = threadIdx.x; u < U; u += NT) cnt[u] = 0;
     __syncthreads();
-#pragma unroll
-    for (int q = 0; q < KEEP; ++q) { const int t = mine[q]; if (t >= 0 && t < V && (int)threadIdx.x + q * NT >= out_start) atomicAdd(&cnt[hist_rank(c, t)], 1u); }
-    for (int j = threadIdx.x + KEEP * NT; j < len; j += NT) {
+    for (int j = threadIdx.x; j < nst; j += NT) {
+        const int t = staged[j];
+        if (t >= 0 && t < V && j >= out_start) atomicAdd(&cnt[hist_rank(c, t)], 1u);
+    }
+    for (int j = threadIdx.x + HIST_STAGED; j < len; j += NT) {
         int t = __ldg(ids + j);
         if (t >= 0 && t < V && j >= out_start) atomicAdd(&cnt[hist_rank(c, t)], 1u);
     }
@@ -1814,15 +1844,23 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         }
     }
     // penalised tokens, straight from the history tables: one distinct id per thread and round,
-    // so that a dense head of the vocabulary does not pile up on a few threads
+    // so that a dense head of the vocabulary does not pile up on a few threads; four rounds at a
+    // time, so that their scattered loads (a round trip each, behind the other rows' streams) overlap
     if (c.has_hist) {
-        for (uint32_t r = threadIdx.x; r < c.n_distinct; r += NT) {
-            const int i = hist_id_of_rank(c, r);
-            const float x = E::load(elem_ptr<DT>(c, i), 0);
-            const uint32_t cntv = c.counts[r];
-            const float av = penalise_counted(c, x, cntv);
-            const uint32_t key = key_of(__fmul_rn(av, c.invT));
-            if (key >= tau_key) cand_append_one(s, cs, comp_of(key, i));
+        constexpr int PG = 4;
+        for (uint32_t r0 = threadIdx.x; r0 < c.n_distinct; r0 += PG * NT) {
+            int id[PG]; float x[PG];
+#pragma unroll
+            for (int u = 0; u < PG; ++u) { const uint32_t r = r0 + u * NT; id[u] = r < c.n_distinct ? hist_id_of_rank(c, r) : -1; }
+#pragma unroll
+            for (int u = 0; u < PG; ++u) x[u] = id[u] >= 0 ? E::load(elem_ptr<DT>(c, id[u]), 0) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < PG; ++u) {
+                if (id[u] < 0) continue;
+                const float av = penalise_counted(c, x[u], c.counts[r0 + u * NT]);
+                const uint32_t key = key_of(__fmul_rn(av, c.invT));
+                if (key >= tau_key) cand_append_one(s, cs, comp_of(key, id[u]));
+            }
         }
     }
     __syncthreads();
@@ -1884,7 +1922,54 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     rg.seg_base = s.seg_base;
     rg.buf = smem + COMMON_BYTES;
     rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
+    // A row that turns out to need the general path waits for the ring's copies before it reuses the
+    // shared memory.
+    // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
+    // stream (the producer of the logits) was still running: wait for it before anything is read or written.
+    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The launch arguments are in constant memory that no SM has seen before this launch: each 64-byte
+    // line of them costs a miss at first touch, and a warp that needs several takes them one after
+    // another.  The lines that only the end of a row needs are touched here once, each from a warp
+    // of its own, so that those misses overlap the stream instead of standing in the row's tail.
+    {
+        uint32_t touch;
+        switch (threadIdx.x >> 5) {
+            case 11: touch = (uint32_t)(uintptr_t)a.seeds; break;
+            case 12: touch = (uint32_t)a.num_top + (uint32_t)a.step; break;
+            case 13: touch = (uint32_t)(uintptr_t)a.out_row_status; break;
+            case 14: touch = (uint32_t)a.backfill_len; break;
+            case 15: touch = (uint32_t)a.elem_size + (uint32_t)a.seg_row_offset; break;
+            default: touch = 1u; break;
+        }
+        if (touch == 0xFFFFFFF1u) s.bcast[3] = touch;      // (never: keeps the reads)
+    }
+    // The row's own parameters and the first part of its history are asked for before the ring is started: a
+    // load issued after the ring's copies (this CTA's and every other's) queues behind megabytes of
+    // them; issued before, it is back within an idle round trip, while thread 0 is still setting up.
+    // With histories the loads come first (the history build waits for them, and so does every thread
+    // at its first barrier); without, they follow the ring start as the first tiles travel, since
+    // reading a dozen more launch arguments first would hold the ring back for nothing.
+    RowParams rp;
     RowCtx c;
+    int o0 = 0, o1 = 0, ostart = 0;
+    const bool with_hist = a.hist_ids && a.hist_off;
+    auto load_params = [&]() {
+        rp.T = a.temperature ? a.temperature[b] : 1.0f;
+        rp.top_k = a.top_k ? a.top_k[b] : 0;
+        rp.top_p = a.top_p ? a.top_p[b] : 1.0f;
+        rp.min_p = a.min_p ? a.min_p[b] : 0.0f;
+        rp.seed = a.seeds ? a.seeds[b] : 0ull;
+        c.r = a.rep ? a.rep[b] : 1.0f;
+        c.p = a.pres ? a.pres[b] : 0.0f;
+        c.f = a.freq ? a.freq[b] : 0.0f;
+    };
+    rp.R = a.row_base + (uint32_t)b;
+    if (with_hist) {
+        load_params();
+        o0 = a.hist_off[b]; o1 = a.hist_off[b + 1];
+        if (a.out_start) ostart = a.out_start[b];
+        if (o1 > o0) hist_prefetch(a.hist_ids + o0, o1 - o0, (int32_t *)smem);
+    }
     c.row = (const char *)a.logits + (size_t)b * (size_t)a.row_stride * Elem<DT>::SIZE;
     c.V = V;
     c.nseg = a.nseg; c.Vs = a.Vs; c.seg_base = s.seg_base;
@@ -1899,29 +1984,9 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
                                                     : (const char *)c.row + (size_t)j * (size_t)a.seg_stride * Elem<DT>::SIZE;
         }
     }
-    // The ring is started before anything else is read, the row's own parameters included: their
-    // loads and the first tiles then travel together.  A row that turns out to need the general
-    // path waits for these copies before it reuses the shared memory.
-    // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
-    // stream (the producer of the logits) was still running: wait for it before anything is read or written.
-    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.wait;" ::: "memory");
-    // The launch arguments are in constant memory that no SM has seen before this launch: each 64-byte
-    // line of them costs a miss at first touch, and a warp that needs several takes them one after
-    // another.  The lines that only the end of a row needs are touched here once, each from a warp
-    // of its own, so that those misses overlap the stream instead of standing in the row's tail.
-    {
-        uint32_t touch;
-        switch (threadIdx.x >> 5) {
-            case 12: touch = (uint32_t)a.num_top + (uint32_t)a.step; break;
-            case 13: touch = (uint32_t)(uintptr_t)a.out_row_status; break;
-            case 14: touch = (uint32_t)a.backfill_len; break;
-            case 15: touch = (uint32_t)a.elem_size + (uint32_t)a.seg_row_offset; break;
-            default: touch = 1u; break;
-        }
-        if (touch == 0xFFFFFFF1u) s.bcast[3] = touch;      // (never: keeps the reads)
-    }
     const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
     if (ring_started) candidate_begin<DT>(s, rg, c);
+    if (!with_hist) load_params();
 
     HistBins h;
     h.cnt = (uint32_t *)smem;
@@ -1934,13 +1999,6 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     hs.coarse = hs.bitmap + (nwords + 1);
     hs.counts = hs.coarse + (ncoarse + 1);
 
-    RowParams rp;
-    rp.T = a.temperature ? a.temperature[b] : 1.0f;
-    rp.top_k = a.top_k ? a.top_k[b] : 0;
-    rp.top_p = a.top_p ? a.top_p[b] : 1.0f;
-    rp.min_p = a.min_p ? a.min_p[b] : 0.0f;
-    rp.seed = a.seeds ? a.seeds[b] : 0ull;
-    rp.R = a.row_base + (uint32_t)b;
     rp.greedy = !(rp.T > 0.0f);
     rp.ln_min_p = (!rp.greedy && rp.min_p > 0.0f) ? log((double)rp.min_p) : 0.0;
 
@@ -1949,21 +2007,14 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     if (rp.T < 0.0f || rp.T != rp.T) out.status |= ALBIREO_ROW_BAD_PARAM;
 
     c.invT = rp.greedy ? 1.0f : __fdiv_rn(1.0f, rp.T);
-    c.r = a.rep ? a.rep[b] : 1.0f;
-    c.p = a.pres ? a.pres[b] : 0.0f;
-    c.f = a.freq ? a.freq[b] : 0.0f;
     c.has_hist = false; c.bitmap = nullptr; c.coarse = nullptr; c.counts = nullptr; c.n_distinct = 0; c.ncoarse = 0;
     if (!(c.r > 0.0f)) out.status |= ALBIREO_ROW_BAD_PARAM;
 
     const bool try_candidates = ring_started && candidate_eligible(rp, V, (a.flags & ALBIREO_FLAG_LOGPROB_FULL_VOCAB) && a.num_top > 0);
-    if (a.hist_ids && a.hist_off) {
-        const int o0 = a.hist_off[b], o1 = a.hist_off[b + 1];
-        if (o1 > o0) {
-            const int ostart = a.out_start ? a.out_start[b] : 0;
-            bool ok = build_history(s, hs, c, a.hist_ids + o0, o1 - o0, ostart, a.ws_counts, a.ws_counts_cap, (int64_t)o0);
-            c.has_hist = ok;
-            if (!ok) out.status |= ALBIREO_ROW_HISTORY_OVERFLOW;
-        }
+    if (o1 > o0) {
+        bool ok = build_history(s, hs, c, a.hist_ids + o0, o1 - o0, ostart, (const int32_t *)smem, a.ws_counts, a.ws_counts_cap, (int64_t)o0);
+        c.has_hist = ok;
+        if (!ok) out.status |= ALBIREO_ROW_HISTORY_OVERFLOW;
     }
 
     // dbg / top-N padding first, the paths overwrite what they produce
