@@ -292,7 +292,12 @@ def measure(args, name, rank, world, dev, *, clocks=None, calls=200, min_region_
     import torch.distributed as dist
     from paper_2606_01927_b200 import binding, workloads as W
 
+    if args.no_graph:
+        calls = min(calls, 20)                   # (profiler runs: few launches beside the timed ones)
     w = W.make(name)
+    if args.rows and args.rows < w.B:
+        w = w.rows(0, args.rows)                 # a smaller case of the same workload (profiler captures)
+        w.name = name
     if args.variant == "f16":
         w = W.as_f16(w)
     elif args.variant == "exp1":
@@ -321,9 +326,15 @@ def measure(args, name, rank, world, dev, *, clocks=None, calls=200, min_region_
         t["backfill_ids"] = torch.zeros(w.backfill_len, dtype=torch.int32, device=dev)
         t["feedback_ring"] = torch.full((2 * w.B,), -1, dtype=torch.int64).pin_memory()
 
+    top_kw = {}
+    if w.num_top:                                  # the workload asks for top-N lists: they are part of the call
+        top_kw = dict(num_top=w.num_top,
+                      out_top_ids=torch.empty((w.B, w.num_top), dtype=torch.int32, device=dev),
+                      out_top_logprobs=torch.empty((w.B, w.num_top), dtype=torch.float32, device=dev))
+
     def step(i, st):
         sampler.albireo_sample(bufs[i % n_rot], **t, out_tokens=out_tok, out_logprobs=out_lp, stream=st,
-                               row_base=w.row_base, flags=flags)
+                               row_base=w.row_base, flags=flags, **top_kw)
 
     def barrier():
         if world > 1:
@@ -551,6 +562,9 @@ def main():
     ap.add_argument("--all-configs", action="store_true",
                     help="also time configs 1-5 and put one compact record per config into `per_config`")
     ap.add_argument("--no-per-config", action="store_true", help="(default run) leave `per_config` out")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="take only the first ROWS rows of the workload: a small case of the same kernel for a profiler "
+                         "capture; a line printed with this flag is not the metric")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -589,6 +603,18 @@ def main():
     e2e = measure_e2e(args, res, rank, world, dev)
     value = world * w.B / (res["ms_per_step"] * 1e-3)
 
+    # the same region with programmatic dependent launch between the calls (each launch's set-up overlaps
+    # the tail of the call before it, as it would overlap the tail of the LM-head GEMM in a decode step):
+    # reported beside the headline, which stays the plain launch
+    pdl_us = None
+    if world == 1 and not args.pdl and not args.no_graph and not args.rows:
+        import copy
+        a2 = copy.copy(args); a2.pdl = True
+        res["bufs"] = None
+        rp = measure(a2, args.workload, rank, world, dev, calls=0, min_region_ms=20.0, ceiling=False)
+        pdl_us = rp["ms_per_step"] * 1e3
+        del rp
+
     per_config = None
     if world == 1 and (args.all_configs or not args.no_per_config):
         peak, peak_src = measured_peak()
@@ -597,7 +623,7 @@ def main():
             if name == args.workload:
                 r = res
             else:
-                del res["bufs"]                      # (one workload's buffers at a time)
+                res["bufs"] = None                   # (one workload's buffers at a time)
                 torch.cuda.empty_cache()
                 r = measure(args, name, rank, world, dev, calls=50, min_region_ms=20.0, ceiling=True)
             wi = r["w"]
@@ -630,7 +656,10 @@ def main():
             },
             "replays": res["replays"], "timed_region_ms": res["elapsed_ms"],
             "tokens_per_s": value,
-            "roofline": roofline_of(w, res, peak, peak_src),
+            "roofline": dict(roofline_of(w, res, peak, peak_src),
+                             **({"programmatic_launch_us": pdl_us,
+                                 "programmatic_launch_frac": algorithmic_bytes(w) / (pdl_us * 1e-6) / 1e9 / peak}
+                                if pdl_us else {})),
             "e2e": e2e,
             "gpu_launches": res["launches"],
             "clocks": res["clock_info"],

@@ -175,7 +175,7 @@ class Sampler:
             pass
 
     def _ext(self, B, dev_type, device, *, row_base=0, row_stride=0, num_top=0, want_counts=False,
-             dbg_cap=0, want_status=False, flags=0):
+             dbg_cap=0, want_status=False, flags=0, out_top_ids=None, out_top_logprobs=None):
         ext = SampleExt()
         ext.struct_size = C.sizeof(SampleExt)
         ext.flags = flags
@@ -185,8 +185,15 @@ class Sampler:
         out = {}
         kw = dict(device=device) if dev_type == "cuda" else dict(pin_memory=True)
         if num_top > 0:
-            out["top_ids"] = torch.empty((B, num_top), dtype=torch.int32, **kw)
-            out["top_logprobs"] = torch.empty((B, num_top), dtype=torch.float32, **kw)
+            if out_top_ids is not None and (out_top_ids.dtype != torch.int32 or out_top_ids.numel() < B * num_top
+                                            or not out_top_ids.is_contiguous()):
+                raise ValueError("out_top_ids must be a contiguous int32 tensor of B * num_top entries")
+            if out_top_logprobs is not None and (out_top_logprobs.dtype != torch.float32 or out_top_logprobs.numel() < B * num_top
+                                                 or not out_top_logprobs.is_contiguous()):
+                raise ValueError("out_top_logprobs must be a contiguous float32 tensor of B * num_top entries")
+            out["top_ids"] = torch.empty((B, num_top), dtype=torch.int32, **kw) if out_top_ids is None else out_top_ids
+            out["top_logprobs"] = (torch.empty((B, num_top), dtype=torch.float32, **kw)
+                                   if out_top_logprobs is None else out_top_logprobs)
             ext.out_top_ids = out["top_ids"].data_ptr()
             ext.out_top_logprobs = out["top_logprobs"].data_ptr()
         if want_counts:
@@ -212,7 +219,9 @@ class Sampler:
                        exp1: Optional[torch.Tensor] = None, backfill_ids: Optional[torch.Tensor] = None,
                        backfill_index: Optional[torch.Tensor] = None, feedback_ring: Optional[torch.Tensor] = None,
                        feedback_head: int = 0, output_start: Optional[torch.Tensor] = None,
-                       segment_tensors=None, segment_row_offset: int = 0) -> SampleOutputs:
+                       segment_tensors=None, segment_row_offset: int = 0,
+                       out_top_ids: Optional[torch.Tensor] = None,
+                       out_top_logprobs: Optional[torch.Tensor] = None) -> SampleOutputs:
         """Device-resident call: all tensors on ``self.device``; asynchronous on ``stream``.
 
         ``exp1`` (float32 ``[B, V]``) replaces the counter-based draw by pre-generated Exp(1)
@@ -242,7 +251,8 @@ class Sampler:
             row_stride = logits.stride(1)
         ext, extra = self._ext(B, "cuda", dev, row_base=row_base, row_stride=0 if row_stride == V else row_stride,
                                num_top=num_top, want_counts=want_counts, dbg_cap=dbg_cap,
-                               want_status=want_status, flags=flags)
+                               want_status=want_status, flags=flags, out_top_ids=out_top_ids,
+                               out_top_logprobs=out_top_logprobs)
         if nseg:
             ext.num_segments = nseg
             ext.segment_stride_elems = logits.stride(0)

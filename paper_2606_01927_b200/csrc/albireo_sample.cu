@@ -1645,8 +1645,10 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         // warm-up on the first NT vectors: the k-th largest of the per-thread maxima (each an
         // unpenalised element of the row, all distinct) is a lower bound of the row's k-th
         // largest score
-        // (a large k needs a larger sample to give a useful bound: then the whole first tile)
-        const int wvecs = (has_topk && k > 64) ? TILE_VECS : 1;
+        // (a large k needs a larger sample to give a useful bound: then the whole first tile; so do
+        // fp32 rows, whose vectors hold half as many elements, and short rows, which have few tiles
+        // over which a loose bound could still be tightened)
+        const int wvecs = (has_topk && (k > 64 || E::PER_VEC < 8 || ntiles <= 6)) ? TILE_VECS : 1;
         bool bad = !mbar_wait(&rg.bar[MAX_STAGES - 1], 0);
         if (wvecs > 1 && !bad) bad = !mbar_wait(&rg.bar[0], 0);
         uint32_t mk = 0;
