@@ -164,6 +164,12 @@ __device__ __forceinline__ u64 mass_fx(float d) {
 
 // ------------------------------------------------------------------ block primitives
 
+// what the general path needs of the launch arguments (see general_path_call)
+struct GenArgs {
+    int32_t *dbg_topk_ids; const float *exp1; int64_t exp1_stride; int32_t *out_top_ids; float *out_top_logprobs;
+    uint64_t step; uint32_t flags; int32_t num_top; int32_t dbg_cap;
+};
+
 struct BlockScratch {
     u64 red[NWARPS];
     u64 red2[NWARPS];
@@ -179,6 +185,7 @@ struct BlockScratch {
     uint32_t issued;             // tiles whose copy has been issued so far
     const char *seg_base[ALBIREO_MAX_SEGMENTS];   // where this row's pieces start (rows in pieces only)
     uint32_t nfin_cap;           // general path: min(#finite scores, ALBIREO_MAX_NUM_TOP + 1), parked here until the list is written
+    GenArgs ga;                  // the general path's copy of the launch arguments it uses
 };
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -948,9 +955,9 @@ __device__ u64 resolve_cut(BlockScratch &s, const HistBins &h, const RowCtx &c, 
     return list_resolve(&s, h.list, n, by_mass, rel, lo, hi, zmax);
 }
 
-template <int DT>
-__device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c, const RowParams &rp,
-                             const SampleArgs &a, int b, RowOut &out) {
+template <int DT, class A>
+__device__ __forceinline__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c, const RowParams &rp,
+                                             const A &a, int b, RowOut &out) {
     const int V = c.V;
     // pass 0: the largest key and the number of finite scores
     uint32_t kbest = 0, nfin_local = 0;
@@ -1178,6 +1185,23 @@ __device__ void general_path(BlockScratch &s, const HistBins &h, const RowCtx &c
     out.n_keep = (int32_t)n_keep;
 
     if (want_top_list) write_top_list(full_lp ? (u64)s.nfin_cap : n_keep, full_lp ? ((u64)KEY_MIN_FINITE << 32) : C2, lnS);
+}
+
+// The general path as a function of its own: its registers are allocated apart from the streaming
+// path's (the whole kernel is held to 64 per thread) and its size does not shape that path's code.
+// The row's context travels by value, the few launch arguments it needs through shared memory
+// (BlockScratch::ga, written by the caller before the barrier in front of the call).
+template <int DT>
+__device__ __noinline__ RowOut general_path_call(BlockScratch *sp, unsigned char *smem, RowCtx c, RowParams rp, int b, uint32_t status) {
+    HistBins h;
+    h.cnt = (uint32_t *)smem;
+    h.limb = (uint32_t *)(smem + HIST_BINS * 4);
+    h.list = (u64 *)(smem + HIST_BINS * 16);
+    h.acc = h.list + GL_CAP;
+    RowOut out;
+    out.token = 0; out.logprob = 0.0f; out.n_keep = 0; out.n_topk = 0; out.status = status;
+    general_path<DT>(*sp, h, c, rp, sp->ga, b, out);
+    return out;
 }
 
 // ------------------------------------------------------------------ TMA bulk-copy ring
@@ -1990,11 +2014,6 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     if (ring_started) candidate_begin<DT>(s, rg, c);
     if (!with_hist) load_params();
 
-    HistBins h;
-    h.cnt = (uint32_t *)smem;
-    h.limb = (uint32_t *)(smem + HIST_BINS * 4);
-    h.list = (u64 *)(smem + HIST_BINS * 16);
-    h.acc = h.list + GL_CAP;
     HistSmem hs;
     const int nwords = (V + 31) >> 5, ncoarse = (nwords + 7) >> 3;
     hs.bitmap = (uint32_t *)((unsigned char *)rg.bar + MAX_STAGES * 8);
@@ -2042,8 +2061,13 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
         if (__syncthreads_or(!landed)) { out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); done = true; }   // the same in every thread
     }
     if (!done) {
+        if (threadIdx.x == 0) {
+            GenArgs &ga = s.ga;
+            ga.dbg_topk_ids = a.dbg_topk_ids; ga.exp1 = a.exp1; ga.exp1_stride = a.exp1_stride; ga.out_top_ids = a.out_top_ids;
+            ga.out_top_logprobs = a.out_top_logprobs; ga.step = a.step; ga.flags = a.flags; ga.num_top = a.num_top; ga.dbg_cap = a.dbg_cap;
+        }
         __syncthreads();
-        general_path<DT>(s, h, c, rp, a, b, out);
+        out = general_path_call<DT>(&s, smem, c, rp, b, out.status);
     }
 
     if (threadIdx.x == 0) {
