@@ -2168,13 +2168,16 @@ size_t history_smem_bytes(int V) {
     size_t nwords = ((size_t)V + 31) / 32, ncoarse = (nwords + 7) / 8;
     return (nwords + 1 + ncoarse + 1 + CNT_CAP) * 4;
 }
-// ring depth: as deep as lets two CTAs share an SM (228 KiB per SM, 1 KiB reserved per CTA)
-int ring_stages_for(int V, bool with_history) {
-    const long budget = (233472 / 2) - 1024 - 1024;      // per CTA: dynamic bytes available
+// ring depth: as deep as lets two CTAs share an SM (228 KiB per SM, 1 KiB reserved per CTA) -- or, for a
+// batch with no more rows than the device has SMs (`alone`: every CTA has an SM to itself), as deep as
+// one CTA's share allows
+int ring_stages_for(int V, bool with_history, bool alone) {
+    const long budget = (alone ? 233472 - 1024 : 233472 / 2 - 1024) - 1024;      // per CTA: dynamic bytes available
     long fixed = COMMON_BYTES + MAX_STAGES * 8 + (with_history ? (long)history_smem_bytes(V) : 0);
     long n = (budget - fixed) / STAGE_BYTES;
+    const long cap = alone ? 6 : 4;
     if (n < 2) n = 2;
-    if (n > 4) n = 4;
+    if (n > cap) n = cap;
     return (int)n;
 }
 size_t smem_bytes_for(int V, bool with_history, int nstages) {
@@ -2298,6 +2301,7 @@ struct albireo_sampler {
     unsigned char *workspace;
     size_t workspace_bytes;
     size_t max_smem;
+    int num_sms;
     uint64_t launches;
     char err[256];
 };
@@ -2351,6 +2355,8 @@ extern "C" int albireo_sample_init(albireo_sampler_t **out, int32_t device, int3
     h->max_history_total = max_history_total;
     h->workspace = (unsigned char *)workspace; h->workspace_bytes = workspace_bytes;
     h->max_smem = smem; h->launches = 0; h->err[0] = 0;
+    h->num_sms = 0;
+    if (cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) { cudaGetLastError(); h->num_sms = 0; }
     *out = h;
     return ALBIREO_OK;
 }
@@ -2391,7 +2397,7 @@ extern "C" int albireo_sample(albireo_sampler_t *h, const void *logits, int32_t 
     int cur = -1;
     if (cudaGetDevice(&cur) != cudaSuccess || cur != h->device) { cudaGetLastError(); set_err(h, "the handle's device is not current%s", ""); return ALBIREO_EINVAL; }
 
-    a.nstages = ring_stages_for(V, history_ids != nullptr);
+    a.nstages = ring_stages_for(V, history_ids != nullptr, B <= h->num_sms);
     size_t smem = smem_bytes_for(V, history_ids != nullptr, a.nstages);
     while (smem > h->max_smem && a.nstages > 2) smem = smem_bytes_for(V, history_ids != nullptr, --a.nstages);
     if (smem > h->max_smem) { set_err(h, "vocabulary too large for the on-chip tables%s", ""); return ALBIREO_EUNSUPPORTED; }
@@ -2508,8 +2514,9 @@ extern "C" int albireo_stream_only(albireo_sampler_t *h, const void *logits, int
     if (B == 0) return ALBIREO_OK;
     if (B < 0 || B > h->max_rows || V < 1 || V > h->max_vocab || !logits || !sink) { set_err(h, "bad arguments%s", ""); return ALBIREO_EINVAL; }
     if (dtype != ALBIREO_F32 && dtype != ALBIREO_BF16 && dtype != ALBIREO_F16) { set_err(h, "unknown dtype%s", ""); return ALBIREO_EINVAL; }
-    const int nstages = ring_stages_for(V, false);
-    const size_t smem = smem_bytes_for(V, false, nstages);
+    int nstages = ring_stages_for(V, false, B <= h->num_sms);
+    size_t smem = smem_bytes_for(V, false, nstages);
+    while (smem > h->max_smem && nstages > 2) smem = smem_bytes_for(V, false, --nstages);
     if (smem > h->max_smem) { set_err(h, "vocabulary too large%s", ""); return ALBIREO_EUNSUPPORTED; }
     cudaStream_t st = (cudaStream_t)stream;
     if (dtype == ALBIREO_F32) albireo_stream_only_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
@@ -2537,6 +2544,7 @@ struct FixedDeviceState {
     bool ready;
     uint32_t *counts;     // device address of g_fixed_counts on that device
     size_t max_smem;
+    int num_sms;
 };
 FixedDeviceState g_fixed_dev[FIXED_MAX_DEVICES];
 std::mutex g_fixed_mutex;
@@ -2560,6 +2568,8 @@ int fixed_setup(int dev, FixedDeviceState **out) {
         if (e != cudaSuccess || !ptr) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e)); }
         const size_t smem = enable_large_smem(dev, &e);
         if (e != cudaSuccess) { cudaGetLastError(); return fixed_fail(ALBIREO_ECUDA, "kernel set-up failed: %s", cudaGetErrorString(e)); }
+        d.num_sms = 0;
+        if (cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); d.num_sms = 0; }
         d.counts = (uint32_t *)ptr; d.max_smem = smem; d.ready = true;
     }
     *out = &d;
@@ -2610,7 +2620,7 @@ extern "C" int albireo_sample_fixed_scratch(const void *logits, int32_t B, int32
     a.ws_counts = d->counts;                       // a device address, from cudaGetSymbolAddress
     a.ws_counts_cap = ALBIREO_FIXED_MAX_HISTORY;
 
-    a.nstages = ring_stages_for(V, history_ids != nullptr);
+    a.nstages = ring_stages_for(V, history_ids != nullptr, B <= d->num_sms);
     size_t smem = smem_bytes_for(V, history_ids != nullptr, a.nstages);
     while (smem > d->max_smem && a.nstages > 2) smem = smem_bytes_for(V, history_ids != nullptr, --a.nstages);
     if (smem > d->max_smem) return fixed_fail(ALBIREO_EUNSUPPORTED, "vocabulary too large for the on-chip tables%s", "");
