@@ -1586,6 +1586,19 @@ __device__ uint32_t warm_select(BlockScratch &s, const CandSmem &cs, uint32_t mk
 // Starts the stream of a row: resets the per-row state, arms the mbarriers and issues the first
 // copies.  Called first thing in the kernel, before the row's parameters are loaded and the history
 // tables built, so that the first tiles arrive meanwhile; a block barrier must follow before any wait.
+// The ring's barriers and the block's bookkeeping: touches shared memory only, so under programmatic
+// dependent launch it runs before the wait for the kernel ahead (thread 0 only).
+__device__ __forceinline__ void ring_setup(BlockScratch &s, const Ring &rg) {
+    if (threadIdx.x != 0) return;
+    for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
+    mbar_init(&rg.bar[MAX_STAGES - 1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0; s.issued = 0;
+    s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
+    for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
+}
+// The first copies of the row (thread 0 only; after ring_setup).
 template <int DT>
 __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c) {
     typedef Elem<DT> E;
@@ -1596,20 +1609,10 @@ __device__ void candidate_begin(BlockScratch &s, const Ring &rg, const RowCtx &c
     const int nvec = (c.V - head) / E::PER_VEC;
     const uint4 *vp = (const uint4 *)((const char *)c.row + (size_t)head * E::SIZE);
     const int ntiles = (nvec + NT * TILE_VECS - 1) / (NT * TILE_VECS);
-    {
-        // the copies first: every cycle before them is a cycle nothing is on its way
-        for (int st = 0; st < rg.nstages; ++st) mbar_init(&rg.bar[st], 1);
-        mbar_init(&rg.bar[MAX_STAGES - 1], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (ntiles > 0) ring_issue_first(rg, vp, nvec);
-        const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
-        for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
-        s.issued = (uint32_t)npre;
-        s.cand_cnt = 0; s.overflow = 0; s.runmax = 0; s.timeout = 0;
-        s.mm_max = 0; s.mm_min = 0xFFFFFFFFu; s.found_digit = 0xFFFFFFFFu; s.maint_at = 0xFFFFFFFFu;
-        for (int q = 0; q < MAX_STAGES; ++q) s.done[q] = 0;
-    }
+    if (ntiles > 0) ring_issue_first(rg, vp, nvec);
+    const int npre = ntiles < rg.nstages ? ntiles : rg.nstages;
+    for (int t = 1; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
+    s.issued = (uint32_t)npre;
 }
 
 // which rows the candidate path takes (decided from the row's parameters alone)
@@ -1950,9 +1953,6 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
     // A row that turns out to need the general path waits for the ring's copies before it reuses the
     // shared memory.
-    // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
-    // stream (the producer of the logits) was still running: wait for it before anything is read or written.
-    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.wait;" ::: "memory");
     // The launch arguments are in constant memory that no SM has seen before this launch: each 64-byte
     // line of them costs a miss at first touch, and a warp that needs several takes them one after
     // another.  The lines that only the end of a row needs are touched here once, each from a warp
@@ -1969,6 +1969,12 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
         }
         if (touch == 0xFFFFFFF1u) s.bcast[3] = touch;      // (never: keeps the reads)
     }
+    const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
+    if (ring_started) ring_setup(s, rg);
+    // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
+    // stream (the producer of the logits) was still running: everything above touched only launch
+    // arguments and shared memory; nothing below is read or written before that kernel has finished.
+    if (a.flags & ALBIREO_FLAG_PROGRAMMATIC_LAUNCH) asm volatile("griddepcontrol.wait;" ::: "memory");
     // The row's own parameters and the first part of its history are asked for before the ring is started: a
     // load issued after the ring's copies (this CTA's and every other's) queues behind megabytes of
     // them; issued before, it is back within an idle round trip, while thread 0 is still setting up.
@@ -2010,7 +2016,6 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
                                                     : (const char *)c.row + (size_t)j * (size_t)a.seg_stride * Elem<DT>::SIZE;
         }
     }
-    const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
     if (ring_started) candidate_begin<DT>(s, rg, c);
     if (!with_hist) load_params();
 
