@@ -65,3 +65,26 @@ def test_rows_keeps_global_row_ids_and_history():
     assert part.B == 3 and part.row_base == 2
     assert (part.history_offsets == np.array([0, 20, 40, 60])).all()
     assert (part.history_ids == w.history_ids[40:100]).all()
+
+
+def test_bench_gpus_n_spawns_one_rank_per_gpu(monkeypatch):
+    """`bench.py --gpus N` run plainly hands itself to torch.distributed.run with N ranks on 127.0.0.1."""
+    import importlib.util
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_under_test", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    seen = {}
+    monkeypatch.setattr(subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "5", "--warmup", "3"])
+    try:
+        bench.spawn_ranks(2)
+    except SystemExit as e:
+        assert e.code == 0
+    cmd = seen["cmd"]
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-6:] == ["--gpus", "2", "--steps", "5", "--warmup", "3"] and cmd[-7].endswith("bench.py")
