@@ -11,6 +11,9 @@ The K timed launches are one CUDA graph, replayed until the timed region lasts a
 that the clock samples fall inside it); `ms_per_step` is the region divided by all its launches.
 The line also carries the spread of isolated cold-L2 calls, the duration of the stream alone in the
 same harness (`roofline.read_ceiling_us`), and one compact record per configuration (`per_config`).
+Calls are launched with programmatic stream serialisation by default (each kernel waits for the one
+ahead of it before it touches memory; only its set-up overlaps that kernel's tail); the figure for
+plain launches is in the same line (`roofline.plain_launch_us`), `--no-pdl` makes it the headline.
 With --gpus N > 1 and no WORLD_SIZE in the environment the N ranks are started here.
 
 N > 1 (launched by torch.distributed.run, one rank per GPU): rows are independent
@@ -556,9 +559,13 @@ def main():
                     help="secondary mode: logits start as per-rank vocabulary shards; time all-to-all + sample + "
                          "gather (a2a), the gather-to-one-rank arrangement it replaces (gather), or the step without an "
                          "exchange: the sampler reads the peers' shards in place from symmetric memory (peer)")
-    ap.add_argument("--pdl", action="store_true",
-                    help="launch every call with programmatic stream serialisation (ALBIREO_FLAG_PROGRAMMATIC_LAUNCH): "
-                         "a call's launch overlaps the tail of the call before it; off by default")
+    ap.add_argument("--pdl", action="store_true", default=True,
+                    help="(default) launch every call with programmatic stream serialisation "
+                         "(ALBIREO_FLAG_PROGRAMMATIC_LAUNCH): a call's set-up overlaps the tail of the kernel ahead of it in "
+                         "the stream, as it would overlap the tail of the LM-head GEMM in a decode step; the kernel waits for "
+                         "that kernel before it touches memory, results are identical")
+    ap.add_argument("--no-pdl", dest="pdl", action="store_false",
+                    help="plain launches; the default run reports this figure too, as roofline.plain_launch_us")
     ap.add_argument("--all-configs", action="store_true",
                     help="also time configs 1-5 and put one compact record per config into `per_config`")
     ap.add_argument("--no-per-config", action="store_true", help="(default run) leave `per_config` out")
@@ -603,16 +610,15 @@ def main():
     e2e = measure_e2e(args, res, rank, world, dev)
     value = world * w.B / (res["ms_per_step"] * 1e-3)
 
-    # the same region with programmatic dependent launch between the calls (each launch's set-up overlaps
-    # the tail of the call before it, as it would overlap the tail of the LM-head GEMM in a decode step):
-    # reported beside the headline, which stays the plain launch
-    pdl_us = None
-    if world == 1 and not args.pdl and not args.no_graph and not args.rows:
+    # the same region with the other launch mode (plain launches when the run uses programmatic dependent
+    # launch, and the other way round), reported beside the headline
+    other_us = None
+    if world == 1 and not args.no_graph and not args.rows:
         import copy
-        a2 = copy.copy(args); a2.pdl = True
+        a2 = copy.copy(args); a2.pdl = not args.pdl
         res["bufs"] = None
         rp = measure(a2, args.workload, rank, world, dev, calls=0, min_region_ms=20.0, ceiling=False)
-        pdl_us = rp["ms_per_step"] * 1e3
+        other_us = rp["ms_per_step"] * 1e3
         del rp
 
     per_config = None
@@ -649,7 +655,8 @@ def main():
             "config": {
                 "workload": describe(w), "rows_per_gpu": w.B, "accum": "f32 element-wise, 2^40 fixed-point masses",
                 "l2": f"{res['n_rot']} rotating logits buffers ({res['n_rot'] * w.logit_bytes / 1e6:.0f} MB per GPU) so no call finds its rows in the 126 MB L2",
-                "launch": f"one CUDA graph of K launches, replayed {res['replays']} times inside the timed region" if res["graph"] else "K launches from the host",
+                "launch": (f"one CUDA graph of K launches, replayed {res['replays']} times inside the timed region" if res["graph"] else "K launches from the host")
+                          + ("; programmatic dependent launch between the calls (plain launches: roofline.plain_launch_us)" if args.pdl else "; plain launches"),
                 "path": "general path forced" if args.general_path else "automatic",
                 "variant": args.variant,
                 "programmatic_launch": bool(args.pdl),
@@ -657,9 +664,10 @@ def main():
             "replays": res["replays"], "timed_region_ms": res["elapsed_ms"],
             "tokens_per_s": value,
             "roofline": dict(roofline_of(w, res, peak, peak_src),
-                             **({"programmatic_launch_us": pdl_us,
-                                 "programmatic_launch_frac": algorithmic_bytes(w) / (pdl_us * 1e-6) / 1e9 / peak}
-                                if pdl_us else {})),
+                             **({("plain_launch_us" if args.pdl else "programmatic_launch_us"): other_us,
+                                 ("plain_launch_frac" if args.pdl else "programmatic_launch_frac"):
+                                     algorithmic_bytes(w) / (other_us * 1e-6) / 1e9 / peak}
+                                if other_us else {})),
             "e2e": e2e,
             "gpu_launches": res["launches"],
             "clocks": res["clock_info"],
