@@ -270,7 +270,10 @@ uint64_t albireo_sample_launch_count(const albireo_sampler_t *h);
  * through the sampler's own shared-memory ring, in the sampler's launch shape, testing every tile
  * against a threshold nothing reaches -- and does nothing else.  Its duration is what the stream
  * alone costs on this GPU at this size; benchmarks report it beside the sampler's.
- *   sink  uint32[B] device: one word per row is written (so that the loads are kept).
+ *   sink  uint32[B] device: one word per row is written (so that the loads are kept): the number of
+ *         (warp, tile) pairs that held a value reaching the threshold -- only +inf does, so 0 for ordinary
+ *         rows --, with bit 31 set if a bounded on-chip wait expired.  Only the 16-byte-aligned middle of a
+ *         row is streamed (what the sampler's ring carries); a ragged head or tail is not looked at.
  * Asynchronous on `stream`; errors as albireo_sample.
  */
 int albireo_stream_only(albireo_sampler_t *h, const void *logits, int32_t B, int32_t V, int32_t dtype,

@@ -418,6 +418,8 @@ template <class P> struct VecTest16 {
         return key_of(__fmul_rn(fmaxf(__low2float(m), __high2float(m)), invT));
     }
     static __device__ __forceinline__ uint4 fill() { const uint32_t f = P::NEG_INF | (P::NEG_INF << 16); return make_uint4(f, f, f, f); }
+    // the raw threshold that only +inf reaches (NEG_INF without its sign bit), packed twice
+    static __device__ __forceinline__ uint32_t pos_inf_threshold() { const uint32_t b = P::NEG_INF & 0x7FFFu; return b | (b << 16); }
     // how many of the vector's elements are -inf
     static __device__ __forceinline__ uint32_t count_neginf(const uint4 &q) {
         const uint32_t f = P::NEG_INF | (P::NEG_INF << 16);
@@ -452,6 +454,7 @@ template <> struct VecTest<ALBIREO_F32> {
     }
     static __device__ __forceinline__ uint32_t vmax_key(const uint4 &q, float invT) { return key_of(vmaxz(q, invT)); }
     static __device__ __forceinline__ uint4 fill() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
+    static __device__ __forceinline__ uint32_t pos_inf_threshold() { return 0x7F800000u; }
     static __device__ __forceinline__ uint32_t count_neginf(const uint4 &q) {
         return (uint32_t)(q.x == 0xFF800000u) + (uint32_t)(q.y == 0xFF800000u) + (uint32_t)(q.z == 0xFF800000u) + (uint32_t)(q.w == 0xFF800000u);
     }
@@ -2135,7 +2138,7 @@ __global__ void __launch_bounds__(NT, 2) albireo_stream_only_kernel(const void *
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const int pvec = 16 * lane + (((threadIdx.x >> 5) + lane) & 15);
-    const uint32_t thr = T::raw_threshold(KEY_POS_INF - 1u, 1.0f);
+    const uint32_t thr = T::pos_inf_threshold();      // only +inf reaches it
     int st = 0; uint32_t parity = 0, cnt = 0;
     for (int tile = 0; tile < ntiles; ++tile) {
         if (*(volatile uint32_t *)&dead == 0u) {

@@ -550,3 +550,32 @@ def test_history_overflow_is_flagged_and_skips_the_penalties(binding, flags):
     assert rep.ok() and not rep.excused, (rep.failures[:3], rep.excused[:3])
     flagged = (g["row_status"] & binding.ROW_HISTORY_OVERFLOW) != 0
     assert flagged.tolist() == [b in over for b in range(B)]
+
+
+# ------------------------------------------------------------------ the stream-only measurement aid
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16, torch.float16])
+def test_stream_only_reads_every_streamed_element(binding, sampler, dtype):
+    """The measurement kernel really moves the rows: a +inf anywhere in the streamed part of a row shows
+    in that row's word, ordinary rows give 0, and no wait expires."""
+    B, V = 6, 70001                                    # several tiles and a ragged end
+    g = torch.Generator(device="cpu").manual_seed(5)
+    x = (torch.randn((B, V), generator=g) * 3).to(dtype)
+    per_vec = 16 // x.element_size()
+    where = {1: 5 * per_vec + 1, 3: V - 40 * per_vec, 4: 3 * 512 * 4 * per_vec + 7}     # first tile, last tile, a middle tile
+    for b, i in where.items():
+        x[b, i] = float("inf")
+    xd = x.to(sampler.device)
+    sink = torch.full((B,), 123, dtype=torch.int32, device=sampler.device)
+    n0 = sampler.launch_count()
+    sampler.albireo_stream_only(xd, sink)
+    torch.cuda.synchronize()
+    got = sink.cpu().numpy().astype(np.int64) & 0xFFFFFFFF
+    assert not (got >> 31).any(), got                  # no expired wait
+    assert [int(v > 0) for v in got] == [int(b in where) for b in range(B)], got
+    assert sampler.launch_count() == n0                # (not a sampling launch)
+    with pytest.raises(ValueError):
+        sampler.albireo_stream_only(xd[:, :100], sink)           # not dense
+    with pytest.raises(binding.AlbireoError):
+        sampler.albireo_stream_only(torch.zeros((2000, 8), dtype=dtype, device=sampler.device),
+                                    torch.zeros(2000, dtype=torch.int32, device=sampler.device))   # more rows than the handle allows
