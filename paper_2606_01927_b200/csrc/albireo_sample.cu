@@ -1956,22 +1956,6 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
     rg.bar = (uint64_t *)(rg.buf + (size_t)a.nstages * STAGE_BYTES);
     // A row that turns out to need the general path waits for the ring's copies before it reuses the
     // shared memory.
-    // The launch arguments are in constant memory that no SM has seen before this launch: each 64-byte
-    // line of them costs a miss at first touch, and a warp that needs several takes them one after
-    // another.  The lines that only the end of a row needs are touched here once, each from a warp
-    // of its own, so that those misses overlap the stream instead of standing in the row's tail.
-    {
-        uint32_t touch;
-        switch (threadIdx.x >> 5) {
-            case 11: touch = (uint32_t)(uintptr_t)a.seeds; break;
-            case 12: touch = (uint32_t)a.num_top + (uint32_t)a.step; break;
-            case 13: touch = (uint32_t)(uintptr_t)a.out_row_status; break;
-            case 14: touch = (uint32_t)a.backfill_len; break;
-            case 15: touch = (uint32_t)a.elem_size + (uint32_t)a.seg_row_offset; break;
-            default: touch = 1u; break;
-        }
-        if (touch == 0xFFFFFFF1u) s.bcast[3] = touch;      // (never: keeps the reads)
-    }
     const bool ring_started = !(a.flags & ALBIREO_FLAG_FORCE_GENERAL);
     if (ring_started) ring_setup(s, rg);
     // Under programmatic dependent launch the CTA may have been scheduled while the kernel ahead in the
