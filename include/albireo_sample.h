@@ -274,10 +274,15 @@ uint64_t albireo_sample_launch_count(const albireo_sampler_t *h);
  *         (warp, tile) pairs that held a value reaching the threshold -- only +inf does, so 0 for ordinary
  *         rows --, with bit 31 set if a bounded on-chip wait expired.  Only the 16-byte-aligned middle of a
  *         row is streamed (what the sampler's ring carries); a ragged head or tail is not looked at.
+ *   drop_tile  -1 for a measurement.  >= 0: the copy of that tile of every row is announced to its
+ *         barrier but never issued, so the bounded wait on it must expire: the rows then report bit 31,
+ *         the copies still in flight are waited for, and the kernel returns normally.  This is how the
+ *         tests exercise the expiry of the ring's bounded waits (the sampler's wait routine, with a bound
+ *         of 2^14 polls instead of 2^20 so that the launch stays short) without anything that hangs or faults.
  * Asynchronous on `stream`; errors as albireo_sample.
  */
 int albireo_stream_only(albireo_sampler_t *h, const void *logits, int32_t B, int32_t V, int32_t dtype,
-                        uint32_t *sink, void *stream);
+                        uint32_t *sink, int32_t drop_tile, void *stream);
 
 /* largest history_total albireo_sample_fixed_scratch accepts (entries of its fixed scratch array) */
 #define ALBIREO_FIXED_MAX_HISTORY (1 << 20)

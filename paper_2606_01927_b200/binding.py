@@ -93,7 +93,7 @@ def _load() -> C.CDLL:
     lib.albireo_sample_fixed_scratch_error.restype = C.c_char_p
     lib.albireo_sample_fixed_scratch_error.argtypes = []
     lib.albireo_stream_only.restype = C.c_int
-    lib.albireo_stream_only.argtypes = [vp, vp, i32, i32, i32, vp, vp]
+    lib.albireo_stream_only.argtypes = [vp, vp, i32, i32, i32, vp, i32, vp]
     return lib
 
 
@@ -302,15 +302,17 @@ class Sampler:
             raise AlbireoError(rc, self.last_error())
         return SampleOutputs(out_tokens, out_logprobs, **extra)
 
-    def albireo_stream_only(self, logits: torch.Tensor, sink: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
-        """Measurement aid: the sampler's stream over ``logits`` ([B, V], dense) and nothing else."""
+    def albireo_stream_only(self, logits: torch.Tensor, sink: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+                            drop_tile: int = -1):
+        """Measurement aid: the sampler's stream over ``logits`` ([B, V], dense) and nothing else.
+        ``drop_tile >= 0`` withholds that tile's copy so that the bounded wait on it expires (bit 31 of the sink words)."""
         B, V = logits.shape
         if not logits.is_contiguous() or sink.dtype != torch.int32 or sink.numel() < B:
             raise ValueError("albireo_stream_only wants dense logits and an int32 sink of B words")
         st = torch.cuda.current_stream(logits.device) if stream is None else stream
         with torch.cuda.device(logits.device):
             rc = LIB.albireo_stream_only(self._handle, C.c_void_p(logits.data_ptr()), B, V, _dtype_code(logits),
-                                         C.c_void_p(sink.data_ptr()), C.c_void_p(st.cuda_stream))
+                                         C.c_void_p(sink.data_ptr()), int(drop_tile), C.c_void_p(st.cuda_stream))
         if rc != OK:
             raise AlbireoError(rc, self.last_error())
 

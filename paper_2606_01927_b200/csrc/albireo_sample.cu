@@ -1237,8 +1237,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (int it = 0; it < WAIT_CAP; ++it) if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int cap = WAIT_CAP) {
+    for (int it = 0; it < cap; ++it) if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
 // global -> shared bulk copy; src and dst 16-byte aligned, bytes a multiple of 16
@@ -2094,12 +2094,12 @@ __global__ void __launch_bounds__(NT, 2) albireo_sample_kernel(const SampleArgs 
 // this GPU at this size; the sampler's own work is the difference.  Writes one word per row so that
 // the loads cannot be dropped.
 template <int DT>
-__global__ void __launch_bounds__(NT, 2) albireo_stream_only_kernel(const void *logits, int V, int64_t row_stride, int nstages, uint32_t *sink) {
+__global__ void __launch_bounds__(NT, 2) albireo_stream_only_kernel(const void *logits, int V, int64_t row_stride, int nstages, uint32_t *sink, int drop_tile) {
     typedef Elem<DT> E;
     typedef VecTest<DT> T;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ uint32_t done[MAX_STAGES];
-    __shared__ uint32_t hits, dead;
+    __shared__ uint32_t hits, dead, issued;
     __shared__ const char *no_pieces[1];
     Ring rg;
     rg.nstages = nstages; rg.vps = 0x7FFFFFFF; rg.seg_base = no_pieces;
@@ -2117,16 +2117,22 @@ __global__ void __launch_bounds__(NT, 2) albireo_stream_only_kernel(const void *
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         const int npre = ntiles < nstages ? ntiles : nstages;
-        for (int t = 0; t < npre; ++t) ring_issue(rg, vp, nvec, t, t);
+        for (int t = 0; t < npre; ++t) {
+            if (t == drop_tile) mbar_expect_tx(&rg.bar[t], 16u);      // announced, never copied: the wait on it must expire
+            else ring_issue(rg, vp, nvec, t, t);
+        }
+        issued = (uint32_t)npre;
     }
     __syncthreads();
+    // with a tile withheld the wait is meant to expire: a smaller bound keeps that launch short
+    const int wait_cap = drop_tile >= 0 ? (1 << 14) : WAIT_CAP;
     const int lane = threadIdx.x & 31;
     const int pvec = 16 * lane + (((threadIdx.x >> 5) + lane) & 15);
     const uint32_t thr = T::pos_inf_threshold();      // only +inf reaches it
     int st = 0; uint32_t parity = 0, cnt = 0;
     for (int tile = 0; tile < ntiles; ++tile) {
         if (*(volatile uint32_t *)&dead == 0u) {
-            if (!mbar_wait(&rg.bar[st], parity)) dead = 1u;        // (bounded: the row is given up, the protocol below goes on)
+            if (!mbar_wait(&rg.bar[st], parity, wait_cap)) dead = 1u;        // (bounded: the row is given up, the protocol below goes on)
             else {
                 const uint4 *stage = (const uint4 *)(rg.buf + (size_t)st * STAGE_BYTES) + pvec;
                 const int vbase = tile * NT * TILE_VECS;
@@ -2145,13 +2151,21 @@ __global__ void __launch_bounds__(NT, 2) albireo_stream_only_kernel(const void *
                 __threadfence_block();
                 if (tile + nstages < ntiles && *(volatile uint32_t *)&dead == 0u) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    ring_issue(rg, vp, nvec, tile + nstages, st);
+                    if (tile + nstages == drop_tile) mbar_expect_tx(&rg.bar[st], 16u);
+                    else ring_issue(rg, vp, nvec, tile + nstages, st);
+                    issued = (uint32_t)(tile + nstages + 1);
                 }
             }
         }
         if (++st == nstages) { st = 0; parity ^= 1u; }
     }
     if (cnt && lane == 0) atomicAdd(&hits, cnt);
+    __syncthreads();
+    if (dead && threadIdx.x == 0) {
+        // a wait expired: the copies still in flight land (bounded waits) before the CTA leaves
+        const int hi = (int)issued, lo = hi - nstages > 0 ? hi - nstages : 0;
+        for (int t = lo; t < hi; ++t) if (t != drop_tile) mbar_wait(&rg.bar[t % nstages], (uint32_t)(t / nstages) & 1u);
+    }
     __syncthreads();
     if (threadIdx.x == 0) sink[blockIdx.x] = hits + (dead << 31);
 }
@@ -2500,7 +2514,7 @@ extern "C" uint64_t albireo_sample_launch_count(const albireo_sampler_t *h) { re
 
 // Launches albireo_stream_only_kernel on the rows of `logits` (dense [B, V], one piece per row): see there.
 extern "C" int albireo_stream_only(albireo_sampler_t *h, const void *logits, int32_t B, int32_t V, int32_t dtype,
-                                   uint32_t *sink, void *stream) {
+                                   uint32_t *sink, int32_t drop_tile, void *stream) {
     if (!h) return ALBIREO_EINVAL;
     h->err[0] = 0;
     if (B == 0) return ALBIREO_OK;
@@ -2511,9 +2525,9 @@ extern "C" int albireo_stream_only(albireo_sampler_t *h, const void *logits, int
     while (smem > h->max_smem && nstages > 2) smem = smem_bytes_for(V, false, --nstages);
     if (smem > h->max_smem) { set_err(h, "vocabulary too large%s", ""); return ALBIREO_EUNSUPPORTED; }
     cudaStream_t st = (cudaStream_t)stream;
-    if (dtype == ALBIREO_F32) albireo_stream_only_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
-    else if (dtype == ALBIREO_BF16) albireo_stream_only_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
-    else albireo_stream_only_kernel<ALBIREO_F16><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink);
+    if (dtype == ALBIREO_F32) albireo_stream_only_kernel<ALBIREO_F32><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink, drop_tile);
+    else if (dtype == ALBIREO_BF16) albireo_stream_only_kernel<ALBIREO_BF16><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink, drop_tile);
+    else albireo_stream_only_kernel<ALBIREO_F16><<<B, NT, smem, st>>>(logits, V, (int64_t)V, nstages, sink, drop_tile);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_err(h, "kernel launch failed: %s", cudaGetErrorString(e)); return ALBIREO_ECUDA; }
     return ALBIREO_OK;

@@ -579,3 +579,22 @@ def test_stream_only_reads_every_streamed_element(binding, sampler, dtype):
     with pytest.raises(binding.AlbireoError):
         sampler.albireo_stream_only(torch.zeros((2000, 8), dtype=dtype, device=sampler.device),
                                     torch.zeros(2000, dtype=torch.int32, device=sampler.device))   # more rows than the handle allows
+
+
+def test_bounded_wait_expires_and_the_context_stays_usable(binding, sampler):
+    """A tile whose copy is announced but never issued: the ring's bounded wait on it runs out, every row
+    reports it (bit 31), the copies in flight are waited for, the kernel returns, and the next launches --
+    the stream alone and a real sampling call -- behave as if nothing had happened."""
+    w = W.config1(B=8, V=32000)
+    t = binding.workload_tensors(w, sampler.device)
+    x = t.pop("logits")
+    sink = torch.zeros(w.B, dtype=torch.int32, device=sampler.device)
+    for drop in (0, 2):                                    # in the first fill of the ring, and in a refill
+        sampler.albireo_stream_only(x, sink, drop_tile=drop)
+        torch.cuda.synchronize()
+        got = sink.cpu().numpy().astype(np.int64) & 0xFFFFFFFF
+        assert ((got >> 31) == 1).all(), (drop, got)
+    sampler.albireo_stream_only(x, sink)
+    torch.cuda.synchronize()
+    assert (sink.cpu().numpy() == 0).all()
+    check(binding, sampler, w)
