@@ -1492,6 +1492,53 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
     if (threadIdx.x >= 32) return;
 
     const u64 *sorted = cs.sorted, *gsc = cs.gsc, *efx = cs.efx;
+    int L8 = L7;
+    int tok;
+    float lp_tok, lnS;
+    if (L7 <= 64) {
+        // The usual case (a kept prefix of at most 64): lane l owns elements 2l and 2l + 1 and fetches
+        // everything it will need of them in one round of shared-memory loads; the cut and the race are
+        // then register work, ballots and shuffles only.  Same arithmetic as the general form below.
+        const int qa = 2 * lane, qb = qa + 1;
+        const bool va = qa < L7, vb = qb < L7;
+        const u64 ea = va ? efx[qa] : 0ull, eb = vb ? efx[qb] : 0ull;
+        const u64 ga = va ? gsc[qa] : 0ull, gb = vb ? gsc[qb] : 0ull;
+        const u64 sa = va ? sorted[qa] : 0ull, sb = vb ? sorted[qb] : 0ull;
+        const u64 s0 = __shfl_sync(0xFFFFFFFFu, sa, 0);
+        const u64 local = ea + eb;
+        u64 incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t2; }
+        const u64 tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        u64 S_fx = tot;
+        if (!rp.greedy && rp.top_p < 1.0f) {
+            double t = ceil((double)rp.top_p * (double)tot);
+            u64 target = t <= 1.0 ? 1ull : (u64)t;
+            if (target > tot) target = tot;
+            // smallest prefix whose mass reaches the target: an element stays while the mass ahead of it is short
+            const u64 ahead_a = incl - local, ahead_b = ahead_a + ea;
+            const uint32_t ka = __ballot_sync(0xFFFFFFFFu, va && ahead_a < target);
+            const uint32_t kb = __ballot_sync(0xFFFFFFFFu, vb && ahead_b < target);
+            L8 = __popc(ka) + __popc(kb);
+            const u64 through = ((L8 - 1) & 1) ? ahead_b + eb : ahead_b;     // mass through this lane's element of that parity
+            S_fx = __shfl_sync(0xFFFFFFFFu, through, (L8 - 1) >> 1);
+        }
+        lnS = logf((float)(full_fx ? full_fx : S_fx) * (1.0f / FX_SCALE));
+        tok = comp_idx(s0);
+        lp_tok = full_fx ? __fsub_rn(unkey((uint32_t)(s0 >> 32)), zmax) - lnS : 0.0f;
+        if (L8 > 1) {
+            // argmax of the race score over the kept prefix (ties: lowest id, via the low word ~id)
+            u64 best = 0, sbest = 0;
+            if (qa < L8 && ga > best) { best = ga; sbest = sa; }
+            if (qb < L8 && gb > best) { best = gb; sbest = sb; }
+            const uint32_t ghi = __reduce_max_sync(0xFFFFFFFFu, (uint32_t)(best >> 32));
+            const uint32_t glo = __reduce_max_sync(0xFFFFFFFFu, (uint32_t)(best >> 32) == ghi ? (uint32_t)best : 0u);
+            const uint32_t who = __ballot_sync(0xFFFFFFFFu, (uint32_t)(best >> 32) == ghi && (uint32_t)best == glo);
+            const u64 sw = __shfl_sync(0xFFFFFFFFu, sbest, __ffs(who) - 1);
+            tok = comp_idx(sw);
+            lp_tok = __fsub_rn(unkey((uint32_t)(sw >> 32)), zmax) - lnS;
+        }
+    } else {
     // Each lane owns a contiguous run of the sorted list.  Masses are fixed point: integer sums are
     // exact, so the prefix sums do not depend on the order of the additions.
     const int per = (L7 + 31) >> 5;
@@ -1502,7 +1549,7 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { u64 t2 = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t2; }
     const u64 tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-    int L8 = L7;
+    L8 = L7;
     u64 S_fx = tot;
     if (!rp.greedy && rp.top_p < 1.0f) {
         double t = ceil((double)rp.top_p * (double)tot);
@@ -1519,9 +1566,9 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         L8 = __reduce_add_sync(0xFFFFFFFFu, cnt);
         S_fx = __shfl_sync(0xFFFFFFFFu, last, (L8 - 1) / per);
     }
-    const float lnS = logf((float)(full_fx ? full_fx : S_fx) * (1.0f / FX_SCALE));
-    int tok = comp_idx(sorted[0]);
-    float lp_tok = full_fx ? __fsub_rn(unkey((uint32_t)(sorted[0] >> 32)), zmax) - lnS : 0.0f;
+    lnS = logf((float)(full_fx ? full_fx : S_fx) * (1.0f / FX_SCALE));
+    tok = comp_idx(sorted[0]);
+    lp_tok = full_fx ? __fsub_rn(unkey((uint32_t)(sorted[0] >> 32)), zmax) - lnS : 0.0f;
     if (L8 > 1) {
         // argmax of the race score over the kept prefix (ties: lowest id, via the low word ~id)
         u64 best = 0; int bestq = 0;
@@ -1532,6 +1579,7 @@ __device__ void final_stage(BlockScratch &s, const CandSmem &cs, int n, int L6, 
         const int wq = __shfl_sync(0xFFFFFFFFu, bestq, __ffs(who) - 1);
         tok = comp_idx(sorted[wq]);
         lp_tok = __fsub_rn(unkey((uint32_t)(sorted[wq] >> 32)), zmax) - lnS;
+    }
     }
     out.token = tok; out.logprob = lp_tok; out.n_keep = L8;
     if (a.num_top > 0) {
