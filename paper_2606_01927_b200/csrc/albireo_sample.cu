@@ -1906,12 +1906,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
         }
         if (++st == rg.nstages) { st = 0; parity ^= 1u; }
     }
-    __syncthreads();
-    if (s.timeout) {
-        ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
-        out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); out.n_keep = 0; out.n_topk = 0;
-        return true;
-    }
+    // No barrier here: a warp that has left the loop only appends (atomic slots, its own threshold),
+    // like the warps still streaming, and no rendezvous can be pending that it has not attended.
     // scalar head and tail of a row that is not 16-byte aligned / not a whole number of vectors
     {
         const int tail0 = head + nvec * E::PER_VEC;
@@ -1945,8 +1941,13 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     }
     __syncthreads();
     int n = (int)s.cand_cnt;
-    const uint32_t ovf = s.overflow;
+    const uint32_t ovf = s.overflow, tmo_end = s.timeout;
     __syncthreads();
+    if (tmo_end) {
+        ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
+        out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); out.n_keep = 0; out.n_topk = 0;
+        return true;
+    }
     if (ovf || n < 1) return false;
 
     const uint32_t kmax = s.runmax;    // the row's largest score is always a candidate
