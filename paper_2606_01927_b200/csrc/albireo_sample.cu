@@ -1942,7 +1942,8 @@ __device__ bool candidate_path(BlockScratch &s, const CandSmem &cs, const Ring &
     __syncthreads();
     int n = (int)s.cand_cnt;
     const uint32_t ovf = s.overflow, tmo_end = s.timeout;
-    __syncthreads();
+    // (no second barrier: nothing below writes these words before a barrier of its own -- the
+    // compaction's -- that every thread reaches only after it has read them here)
     if (tmo_end) {
         ring_drain(rg, max(0, (int)s.issued - rg.nstages), (int)s.issued);
         out.status |= ALBIREO_ROW_TIMEOUT; out.token = -1; out.logprob = __uint_as_float(0x7FC00000u); out.n_keep = 0; out.n_topk = 0;
