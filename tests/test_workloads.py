@@ -88,3 +88,27 @@ def test_bench_gpus_n_spawns_one_rank_per_gpu(monkeypatch):
     assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
     assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
     assert cmd[-6:] == ["--gpus", "2", "--steps", "5", "--warmup", "3"] and cmd[-7].endswith("bench.py")
+
+
+def test_bench_helpers_percentile_traffic_and_bytes():
+    """The small pure functions behind the bench line: percentiles, the ncu traffic data file, algorithmic bytes."""
+    import importlib.util
+    import json
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_under_test2", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    xs = [5.0, 1.0, 3.0, 2.0, 4.0]
+    assert bench.percentile(xs, 0.0) == 1.0 and bench.percentile(xs, 1.0) == 5.0 and bench.percentile(xs, 0.5) == 3.0
+    assert abs(bench.percentile(xs, 0.1) - 1.4) < 1e-12 and bench.percentile([], 0.5) is None
+    data = json.load(open(os.path.join(root, "profiles", "ncu_traffic.json")))
+    for name, rec in data.items():
+        assert bench.ncu_traffic(name) == rec["dram_bytes_per_launch"]
+        assert os.path.exists(os.path.join(root, rec["source"]))
+        w = W.make(name)
+        # captured DRAM traffic is the algorithmic bytes plus a few per cent at most: every logit is read once
+        assert 1.0 <= rec["dram_bytes_per_launch"] / bench.algorithmic_bytes(w) < 1.03, name
+    assert bench.ncu_traffic("no-such-workload") is None
+    w = W.make("configM")
+    assert bench.algorithmic_bytes(w) == w.B * w.V * 2 + w.B * (4 * 3 + 16)      # logits + T, top_k, top_p + seed + outputs
